@@ -1,0 +1,155 @@
+/*
+ * arrol.h - C ABI of the B200 (sm_100a) prune-and-rebatch library for online rollout pruning.
+ *
+ * The four compute calls follow the method's problem statement:
+ *   arrol_score_partial  quality head on the policy's hidden state at the detection length, score -> [0,1]
+ *                        -> binned posterior                      (Section 4.2; Appendix A.4)
+ *   arrol_select         per-group correctness-balancing selection, exactly K of G kept
+ *                                                                  (Section 4.1, Theorem 1's rule)
+ *   arrol_compact        filter pruned rollouts and re-batch the survivors, with group-relative
+ *                        advantages on the survivors               (Section 4.3 (ii); Algorithm 1; Section 3)
+ *   arrol_token_logprob  selected-token log-probability of every survivor token from the lm_head,
+ *                        vocabulary-chunked, logits never stored   (Section 3; Algorithm 1 "log-probs on R'")
+ *
+ * Conventions for every call unless a parameter says otherwise:
+ *   - Pointers are DEVICE pointers owned by the caller.  The library keeps no reference to them once the
+ *     call's work has completed on `stream`, never frees them, and allocates nothing after arrol_create.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls are asynchronous:
+ *     the return value reports argument validation and launch errors only.  Conditions found on the device
+ *     (destination too small, target id outside the vocabulary, a bounded wait that ran out) are recorded in
+ *     a status word and read with arrol_poll_status; the device never traps.
+ *   - Return value: ARROL_OK (0) or a negative arrol_status.
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x arrol_create fails.
+ */
+#ifndef ARROL_H_
+#define ARROL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct arrol_ctx arrol_ctx; /* opaque: device id, SM count, status word, small scratch */
+
+typedef enum { ARROL_F32 = 0, ARROL_BF16 = 1 } arrol_dtype;
+
+typedef enum {
+    ARROL_OK = 0,
+    ARROL_ERR_INVALID_ARG = -1,   /* NULL where data is required, negative size, misaligned pointer/stride */
+    ARROL_ERR_UNSUPPORTED = -2,   /* valid but outside the supported range (G > 32, d not a multiple of 8, ...) */
+    ARROL_ERR_WORKSPACE = -3,     /* workspace missing or smaller than arrol_token_logprob_workspace says */
+    ARROL_ERR_CAPACITY = -4,      /* device: survivors need more than dst_capacity_tokens rows */
+    ARROL_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed */
+    ARROL_ERR_DEVICE_STATUS = -6, /* device: target id >= V, or an internal bounded wait expired */
+    ARROL_ERR_NO_DEVICE = -7      /* no usable sm_100 device */
+} arrol_status;
+
+/* Device status bits accumulated in the context's status word (see arrol_poll_status). */
+#define ARROL_DEV_CAPACITY 1u      /* arrol_compact: T > dst_capacity_tokens, nothing was gathered */
+#define ARROL_DEV_BAD_TARGET 2u    /* arrol_token_logprob: a target id >= V (its logp is set to 0) */
+#define ARROL_DEV_WAIT_EXPIRED 4u  /* arrol_token_logprob: a pipeline wait hit its iteration limit */
+
+int arrol_version(void);                    /* major*10000 + minor*100 + patch */
+const char* arrol_status_string(int status); /* static string, never NULL */
+
+/* Creates a context on CUDA device `device` (made current for the calling thread during the call).
+ * Allocates the context's device status word and a small scratch buffer; nothing is allocated later. */
+int arrol_create(arrol_ctx** out, int device);
+int arrol_destroy(arrol_ctx* ctx);
+
+/* Waits for `stream`, copies the device status word to *dev_status_bits (host pointer, may be NULL),
+ * clears it, and returns ARROL_OK if it was 0, else ARROL_ERR_CAPACITY / ARROL_ERR_DEVICE_STATUS. */
+int arrol_poll_status(arrol_ctx* ctx, void* stream, uint32_t* dev_status_bits);
+
+/* ---- Binned posterior table: host helpers (Appendix A.4).  All pointers are HOST pointers. ----------
+ * arrol_calib_counts: c_b^+ / c_b^- = number of historical positive / negative rollouts whose normalised
+ *   score s' falls in bin b(s') = min(B-1, floor(B s')).  sprime [n] in [0,1], y [n] in {0,1}.
+ * arrol_build_q_lut: Laplace-smoothed likelihoods P(b|Y) = (c_b + alpha) / (sum c + alpha B) and the Bayes
+ *   posterior q_b = pi P(b|1) / (pi P(b|1) + (1-pi) P(b|0)), pi = n+/(n+ + n-) (0.5 when both are empty),
+ *   computed in double and rounded once to float.  q_lut [B] is what arrol_score_partial consumes. */
+int arrol_calib_counts(const double* sprime, const uint8_t* y, int64_t n, int B, int64_t* cpos, int64_t* cneg);
+int arrol_build_q_lut(const int64_t* cpos, const int64_t* cneg, int B, double alpha, float* q_lut);
+
+/* ---- Quality head (Section 4.2 "Quality Score Prediction"; Appendix A.4) --------------------------- */
+typedef struct arrol_head {
+    int32_t d;       /* hidden width; multiple of 8                                                    */
+    int32_t h;       /* 0: linear head d -> 1.  > 0: d -> h -> 1 with exact (erf) GELU; multiple of 4  */
+    int32_t dtype;   /* arrol_dtype of hidden, W1, b1, w2, b2                                          */
+    int32_t reserved;
+    const void* W1;  /* device [h, d] row-major; [d] when h == 0                                        */
+    const void* b1;  /* device [h] or NULL (= 0); when h == 0: [1] bias or NULL                          */
+    const void* w2;  /* device [h]; ignored when h == 0                                                 */
+    const void* b2;  /* device [1] or NULL; ignored when h == 0                                         */
+} arrol_head;
+
+typedef struct arrol_calib {
+    int32_t B;          /* number of bins (128 in the paper); ignored when q_lut == NULL                 */
+    int32_t reserved;
+    const float* q_lut; /* device [B] posterior per bin, or NULL: q = sigmoid(score)                     */
+} arrol_calib;
+
+/* For each rollout i < N: x = row row_index[i] (row i when row_index is NULL) of `hidden`
+ * ([rows, row_stride_elems] row-major, head->dtype, 16-byte aligned rows);
+ *   score[i] = head(x);  prob[i] = s' = 1 / (1 + exp(-score[i]));
+ *   bin[i] = min(B-1, floor(B s'));  q[i] = q_lut[bin[i]]   (q[i] = s' when there is no table).
+ * Outputs: score, prob, q float [N] (required); bin int32 [N] or NULL.  fp32 accumulation.
+ * row_index holds int64 row numbers; it must stay valid until the work completes.
+ * Errors: INVALID_ARG for NULL/negative/misaligned arguments, UNSUPPORTED for d % 8 != 0, h % 4 != 0,
+ * h > 4096, or N larger than the context scratch allows for the MLP head (65536). N == 0 is a no-op. */
+int arrol_score_partial(arrol_ctx* ctx, const void* hidden, int64_t row_stride_elems, const int64_t* row_index,
+                        int32_t N, const arrol_head* head, const arrol_calib* calib, float* score, float* prob,
+                        int32_t* bin, float* q, void* stream);
+
+/* ---- Per-group selection (Section 4.1; Theorem 1: j^ = argmin_j |mu_{-j} - rho|) -------------------
+ * q [P*G] float, group-major (rollouts of prompt p are q[p*G .. p*G+G-1]).  For each group, while more than
+ * K members remain (n of them, sum Sigma): remove the member minimising |q_j - (Sigma - rho (n-1))|, which
+ * is the member whose removal leaves the group mean closest to rho; of equal candidates the one with the
+ * highest index is removed, so the lower index survives.  Keys are evaluated in double, one rounding per
+ * operation, so the result is reproducible bit for bit.  keep [P*G] uint8 receives 1 (kept) / 0 (pruned).
+ * mode must be 0.  Supported: 1 <= K <= G <= 32.  q must be finite.  P == 0 is a no-op. */
+int arrol_select(arrol_ctx* ctx, const float* q, int32_t P, int32_t G, int32_t K, double rho, int32_t mode,
+                 uint8_t* keep, void* stream);
+
+/* ---- Filter + re-batch with advantages (Section 4.3 (ii); Algorithm 1; Section 3) -------------------
+ * Inputs:  keep [N] uint8; lengths [N] int32 (tokens of rollout i, >= 0); src_tok_off [N] int64 (first source
+ *   row of rollout i); src_tokens int32 [source rows] or NULL; src_rows [source rows, row_bytes] or NULL
+ *   (opaque payload per token, e.g. a hidden-state row; row_bytes a multiple of 16, base 16-byte aligned);
+ *   rewards [N] float; G = group size (N % G == 0).
+ * Outputs: survivor_idx [<= N] int32, ascending original indices of kept rollouts (S of them);
+ *   cu_seqlens [<= N+1] int64, exclusive prefix sum of the survivors' lengths (cu_seqlens[S] = T);
+ *   d_num [2] int64 = {S, T};  adv [<= N] float, A = (R - mean) / (std + eps) over the kept rollouts of the
+ *   survivor's group, std with divisor (n - ddof) (0 when n - ddof <= 0; exactly 0 when all kept rewards of
+ *   the group are equal);  dst_tokens [cap] / dst_rows [cap, row_bytes]: row cu_seqlens[s] + t receives source
+ *   row src_tok_off[survivor_idx[s]] + t;  tok_adv [cap] float or NULL: adv of the token's rollout;
+ *   tok_seq [cap] int32 or NULL: survivor ordinal s of the token.   cap = dst_capacity_tokens.
+ * If T > dst_capacity_tokens the scan outputs (survivor_idx, cu_seqlens, d_num, adv) are still written, nothing
+ * is gathered, and ARROL_DEV_CAPACITY is recorded.  T never leaves the device: no host synchronisation.
+ * dst_* may be NULL when the matching src_* is NULL. */
+int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths, const int64_t* src_tok_off,
+                  int32_t N, int32_t G, const int32_t* src_tokens, const void* src_rows, int32_t row_bytes,
+                  const float* rewards, float eps, int32_t ddof, int64_t dst_capacity_tokens, int32_t* dst_tokens,
+                  void* dst_rows, int64_t* cu_seqlens, int32_t* survivor_idx, float* adv, float* tok_adv,
+                  int32_t* tok_seq, int64_t* d_num, void* stream);
+
+/* ---- Selected-token log-probability (Section 3: log pi_theta(o_t | o_<t); Algorithm 1) -------------
+ * hidden [T_max, d] bf16 row-major; W_vocab [V, d] bf16 row-major (the layout of an nn.Linear / tied
+ * embedding weight); targets [T_max] int32.  T = min(*d_T, T_max) when d_T != NULL (device int64), else T_max.
+ * For t < T:  z_v = inv_temperature * sum_k hidden[t,k] W_vocab[v,k]  (bf16 products, fp32 accumulation on
+ * the tensor cores);  lse[t] = log sum_v exp z_v (running max / sum over vocabulary chunks, fp32);
+ * logp[t] = z_{targets[t]} - lse[t].  targets[t] < 0 marks an ignored position: logp[t] = 0.  A target >= V sets
+ * logp[t] = 0 and records ARROL_DEV_BAD_TARGET.  Rows t >= T of the outputs are not written.
+ * logp float [T_max]; lse float [T_max] or NULL.  Both pointers 16-byte aligned; d % 8 == 0; inv_temperature > 0.
+ * workspace: device scratch of at least arrol_token_logprob_workspace(ctx, T_max, d, V) bytes, 256-byte
+ * aligned (holds per-split running maxima / sums when the vocabulary is split across thread blocks); its
+ * contents need not be initialised and are undefined afterwards. */
+size_t arrol_token_logprob_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
+int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                        int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
+                        float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ARROL_H_ */

@@ -1,0 +1,221 @@
+"""ctypes binding of libarrol.so: argument marshalling only, same names as the C ABI (include/arrol.h).
+
+torch supplies device memory and the current stream; every step of the path runs in the library's CUDA
+kernels.  There is no fallback: if the library is missing or no sm_100 device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libarrol.so")
+
+ARROL_F32, ARROL_BF16 = 0, 1
+DEV_CAPACITY, DEV_BAD_TARGET, DEV_WAIT_EXPIRED = 1, 2, 4
+
+EXPORTS = [
+    "arrol_version", "arrol_status_string", "arrol_create", "arrol_destroy", "arrol_poll_status",
+    "arrol_calib_counts", "arrol_build_q_lut", "arrol_score_partial", "arrol_select", "arrol_compact",
+    "arrol_token_logprob_workspace", "arrol_token_logprob",
+]
+
+
+class ArrolError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s failed: %s (%d)" % (where, status_string(code), code))
+
+
+class _Head(C.Structure):
+    _fields_ = [("d", C.c_int32), ("h", C.c_int32), ("dtype", C.c_int32), ("reserved", C.c_int32),
+                ("W1", C.c_void_p), ("b1", C.c_void_p), ("w2", C.c_void_p), ("b2", C.c_void_p)]
+
+
+class _Calib(C.Structure):
+    _fields_ = [("B", C.c_int32), ("reserved", C.c_int32), ("q_lut", C.c_void_p)]
+
+
+_lib = None
+
+
+def load_library():
+    """Loads libarrol.so; raises if it has not been built (python -m paper_2603_24840_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError("%s not found: build it with `python paper_2603_24840_b200/build.py` "
+                                "(there is no CPU or PyTorch fallback)" % LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
+    lib.arrol_version.restype = C.c_int
+    lib.arrol_status_string.restype = C.c_char_p
+    lib.arrol_status_string.argtypes = [C.c_int]
+    lib.arrol_create.argtypes = [C.POINTER(C.c_void_p), C.c_int]
+    lib.arrol_destroy.argtypes = [C.c_void_p]
+    lib.arrol_poll_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
+    lib.arrol_calib_counts.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_void_p, C.c_void_p]
+    lib.arrol_build_q_lut.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_double, C.c_void_p]
+    lib.arrol_score_partial.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32,
+                                        C.POINTER(_Head), C.POINTER(_Calib), C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_void_p]
+    lib.arrol_select.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_double, C.c_int32,
+                                 C.c_void_p, C.c_void_p]
+    lib.arrol_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                  C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_float, C.c_int32, C.c_int64,
+                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                  C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.arrol_token_logprob_workspace.restype = C.c_size_t
+    lib.arrol_token_logprob_workspace.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32]
+    lib.arrol_token_logprob.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                        C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_size_t, C.c_void_p]
+    for fn in ("arrol_create", "arrol_destroy", "arrol_poll_status", "arrol_calib_counts", "arrol_build_q_lut",
+               "arrol_score_partial", "arrol_select", "arrol_compact", "arrol_token_logprob"):
+        getattr(lib, fn).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().arrol_status_string(int(code)).decode()
+
+
+def arrol_version() -> int:
+    return int(load_library().arrol_version())
+
+
+def _check(code: int, where: str):
+    if code != 0:
+        raise ArrolError(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return ARROL_F32
+    if t.dtype == torch.bfloat16:
+        return ARROL_BF16
+    raise TypeError("hidden / head tensors are float32 or bfloat16")
+
+
+class Context:
+    """Owns an arrol_ctx on one CUDA device."""
+
+    def __init__(self, device: int = 0):
+        lib = load_library()
+        self._h = C.c_void_p()
+        _check(lib.arrol_create(C.byref(self._h), int(device)), "arrol_create")
+        self.device = int(device)
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            load_library().arrol_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._h
+
+
+def arrol_poll_status(ctx: Context, stream=None, raise_on_error: bool = True) -> int:
+    bits = C.c_uint32(0)
+    rc = load_library().arrol_poll_status(ctx.handle, _stream(stream), C.byref(bits))
+    if rc != 0 and raise_on_error:
+        raise ArrolError(rc, "arrol_poll_status (device bits = %d)" % bits.value)
+    return int(bits.value)
+
+
+def arrol_calib_counts(sprime, y, B: int):
+    """Host helper: histogram counts of historical scores per bin (numpy in, numpy out)."""
+    import numpy as np
+    sprime = np.ascontiguousarray(sprime, dtype=np.float64)
+    y = np.ascontiguousarray(y, dtype=np.uint8)
+    cpos = np.empty(B, dtype=np.int64)
+    cneg = np.empty(B, dtype=np.int64)
+    _check(load_library().arrol_calib_counts(sprime.ctypes.data, y.ctypes.data, sprime.shape[0], int(B),
+                                             cpos.ctypes.data, cneg.ctypes.data), "arrol_calib_counts")
+    return cpos, cneg
+
+
+def arrol_build_q_lut(cpos, cneg, alpha: float = 1.0):
+    """Host helper: posterior per bin as float32 numpy [B]."""
+    import numpy as np
+    cpos = np.ascontiguousarray(cpos, dtype=np.int64)
+    cneg = np.ascontiguousarray(cneg, dtype=np.int64)
+    B = cpos.shape[0]
+    q = np.empty(B, dtype=np.float32)
+    _check(load_library().arrol_build_q_lut(cpos.ctypes.data, cneg.ctypes.data, int(B), float(alpha),
+                                            q.ctypes.data), "arrol_build_q_lut")
+    return q
+
+
+def arrol_score_partial(ctx: Context, hidden: torch.Tensor, head: dict, N: int, score: torch.Tensor,
+                        prob: torch.Tensor, q: torch.Tensor, bin: Optional[torch.Tensor] = None,
+                        row_index: Optional[torch.Tensor] = None, q_lut: Optional[torch.Tensor] = None,
+                        row_stride: Optional[int] = None, stream=None):
+    """head = {"W1", "b1", "w2", "b2", "h"} (device tensors or None).  Outputs are written in place."""
+    hs = _Head()
+    hs.d = hidden.shape[-1]
+    hs.h = int(head.get("h", 0))
+    hs.dtype = _dtype_code(hidden)
+    for name in ("W1", "b1", "w2", "b2"):
+        t = head.get(name)
+        if t is not None and t.dtype != hidden.dtype:
+            raise TypeError("head tensors share the hidden dtype")
+        setattr(hs, name, None if t is None else t.data_ptr())
+    cs = _Calib()
+    cs.B = 0 if q_lut is None else q_lut.shape[0]
+    cs.q_lut = None if q_lut is None else q_lut.data_ptr()
+    stride = hidden.stride(-2) if row_stride is None else int(row_stride)
+    _check(load_library().arrol_score_partial(ctx.handle, _ptr(hidden), stride, _ptr(row_index), int(N),
+                                              C.byref(hs), C.byref(cs), _ptr(score), _ptr(prob), _ptr(bin),
+                                              _ptr(q), _stream(stream)), "arrol_score_partial")
+
+
+def arrol_select(ctx: Context, q: torch.Tensor, P: int, G: int, K: int, rho: float, keep: torch.Tensor,
+                 mode: int = 0, stream=None):
+    _check(load_library().arrol_select(ctx.handle, _ptr(q), int(P), int(G), int(K), float(rho), int(mode),
+                                       _ptr(keep), _stream(stream)), "arrol_select")
+
+
+def arrol_compact(ctx: Context, keep, lengths, src_tok_off, N: int, G: int, rewards, dst_capacity_tokens: int,
+                  cu_seqlens, survivor_idx, adv, d_num, src_tokens=None, dst_tokens=None, src_rows=None,
+                  dst_rows=None, row_bytes: int = 0, tok_adv=None, tok_seq=None, eps: float = 1e-6, ddof: int = 0,
+                  stream=None):
+    _check(load_library().arrol_compact(ctx.handle, _ptr(keep), _ptr(lengths), _ptr(src_tok_off), int(N), int(G),
+                                        _ptr(src_tokens), _ptr(src_rows), int(row_bytes), _ptr(rewards),
+                                        float(eps), int(ddof), int(dst_capacity_tokens), _ptr(dst_tokens),
+                                        _ptr(dst_rows), _ptr(cu_seqlens), _ptr(survivor_idx), _ptr(adv),
+                                        _ptr(tok_adv), _ptr(tok_seq), _ptr(d_num), _stream(stream)),
+           "arrol_compact")
+
+
+def arrol_token_logprob_workspace(ctx: Context, T_max: int, d: int, V: int) -> int:
+    return int(load_library().arrol_token_logprob_workspace(ctx.handle, int(T_max), int(d), int(V)))
+
+
+def arrol_token_logprob(ctx: Context, hidden, W_vocab, targets, T_max: int, d: int, V: int, logp, workspace,
+                        lse=None, d_T=None, inv_temperature: float = 1.0, stream=None):
+    _check(load_library().arrol_token_logprob(ctx.handle, _ptr(hidden), _ptr(W_vocab), _ptr(targets), int(T_max),
+                                              _ptr(d_T), int(d), int(V), float(inv_temperature), _ptr(logp),
+                                              _ptr(lse), _ptr(workspace),
+                                              0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                              _stream(stream)), "arrol_token_logprob")

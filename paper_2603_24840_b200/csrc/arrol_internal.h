@@ -1,0 +1,46 @@
+// Internal declarations shared by the library's translation units (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "arrol.h"
+
+struct arrol_ctx {
+    int device;
+    int sm_count;
+    uint32_t* d_status;        // device status word (bits ARROL_DEV_*)
+    uint32_t* h_status;        // pinned host mirror used by arrol_poll_status
+    float* d_scratch;          // MLP-head partial sums: [ARROL_SCRATCH_FLOATS]
+    void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
+};
+
+constexpr int ARROL_MAX_MLP_N = 65536;       // rollouts per arrol_score_partial call with an MLP head
+constexpr int ARROL_MLP_TH = 64;             // hidden units per MLP thread-block tile
+constexpr int ARROL_MAX_H = 4096;
+constexpr size_t ARROL_SCRATCH_FLOATS = (size_t)ARROL_MAX_MLP_N * (ARROL_MAX_H / ARROL_MLP_TH);
+
+#define ARROL_CUDA_OK(expr)                      \
+    do {                                         \
+        cudaError_t e__ = (expr);                \
+        if (e__ != cudaSuccess) {                \
+            (void)cudaGetLastError();            \
+            return ARROL_ERR_CUDA;               \
+        }                                        \
+    } while (0)
+
+static inline bool arrol_aligned(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+// Device guard: makes the context's device current for the duration of a call.
+struct ArrolDeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit ArrolDeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        cur = dev;
+    }
+    ~ArrolDeviceGuard() {
+        if (prev >= 0 && prev != cur) (void)cudaSetDevice(prev);
+    }
+    int cur = -1;
+};

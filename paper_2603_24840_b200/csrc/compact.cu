@@ -1,0 +1,208 @@
+// arrol_compact: filter pruned rollouts and re-batch the survivors (Section 4.3 (ii); Algorithm 1), with the
+// group-relative advantage evaluated on the survivors (Section 3).
+//
+// Kernel 1 (one block): stable partition by a block-wide prefix sum over (kept flag, kept length):
+//   survivor_idx, cu_seqlens, {S, T}, and per-survivor advantages (fp64 statistics over the kept rollouts of
+//   the group, in index order, rounded once to fp32).
+// Kernel 2 (persistent grid): moves the survivors' rows.  A tile is a run of consecutive destination rows;
+//   one thread per row finds its survivor by binary search in cu_seqlens and writes the per-token outputs
+//   (token id, survivor ordinal, advantage); then the whole block streams the row payload with 16-byte
+//   loads/stores.  T is read from device memory, so there is no host synchronisation between the kernels.
+#include "arrol_internal.h"
+
+namespace {
+
+constexpr int SCAN_THREADS = 1024;
+
+__global__ void __launch_bounds__(SCAN_THREADS)
+scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ lengths, int N, int G,
+                const float* __restrict__ rewards, double eps, int ddof, int64_t capacity,
+                int32_t* __restrict__ survivor_idx, int64_t* __restrict__ cu_seqlens, float* __restrict__ adv,
+                int64_t* __restrict__ d_num, uint32_t* __restrict__ d_status) {
+    __shared__ int32_t warp_cnt[32];
+    __shared__ int64_t warp_tok[32];
+    __shared__ int32_t carry_cnt;
+    __shared__ int64_t carry_tok;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { carry_cnt = 0; carry_tok = 0; cu_seqlens[0] = 0; }
+    __syncthreads();
+
+    for (int base = 0; base < N; base += SCAN_THREADS) {
+        const int i = base + threadIdx.x;
+        const bool kept = (i < N) && keep[i] != 0;
+        int32_t c = kept ? 1 : 0;
+        int64_t t = kept ? (int64_t)max(lengths[i], 0) : 0;
+        // inclusive scan inside the warp
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t oc = __shfl_up_sync(0xffffffffu, c, o);
+            const int64_t ot = __shfl_up_sync(0xffffffffu, t, o);
+            if (lane >= o) { c += oc; t += ot; }
+        }
+        if (lane == 31) { warp_cnt[wid] = c; warp_tok[wid] = t; }
+        __syncthreads();
+        if (wid == 0) {
+            int32_t wc = warp_cnt[lane];
+            int64_t wt = warp_tok[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t oc = __shfl_up_sync(0xffffffffu, wc, o);
+                const int64_t ot = __shfl_up_sync(0xffffffffu, wt, o);
+                if (lane >= o) { wc += oc; wt += ot; }
+            }
+            warp_cnt[lane] = wc;   // inclusive over warps
+            warp_tok[lane] = wt;
+        }
+        __syncthreads();
+        const int32_t cnt_before = carry_cnt + (wid ? warp_cnt[wid - 1] : 0);
+        const int64_t tok_before = carry_tok + (wid ? warp_tok[wid - 1] : 0);
+        if (kept) {
+            const int32_t pos = cnt_before + c - 1;        // survivor ordinal
+            survivor_idx[pos] = i;
+            cu_seqlens[pos + 1] = tok_before + t;
+            // statistics over the kept rollouts of this rollout's group (Section 3, on survivors)
+            const int g0 = (i / G) * G;
+            const int g1 = min(g0 + G, N);
+            int n = 0;
+            double sum = 0.0;
+            for (int r = g0; r < g1; ++r)
+                if (keep[r]) { sum += (double)rewards[r]; ++n; }
+            const double mean = sum / (double)n;
+            double ss = 0.0;
+            for (int r = g0; r < g1; ++r)
+                if (keep[r]) { const double dv = (double)rewards[r] - mean; ss += dv * dv; }
+            double a = 0.0;
+            if (n - ddof > 0) a = ((double)rewards[i] - mean) / (sqrt(ss / (double)(n - ddof)) + eps);
+            adv[pos] = (float)a;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) { carry_cnt += warp_cnt[31]; carry_tok += warp_tok[31]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        d_num[0] = carry_cnt;
+        d_num[1] = carry_tok;
+        if (carry_tok > capacity) atomicOr(d_status, ARROL_DEV_CAPACITY);
+    }
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+constexpr int GATHER_THREADS = 256;
+constexpr int MAX_TILE_ROWS = 256;
+
+// tile_rows: destination rows per tile (<= MAX_TILE_ROWS); vec_per_row = row_bytes / 16 (0 without payload)
+__global__ void __launch_bounds__(GATHER_THREADS)
+gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_seqlens,
+              const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
+              const int32_t* __restrict__ src_tokens, const uint4* __restrict__ src_rows, int vec_per_row,
+              const float* __restrict__ adv, int64_t capacity, int tile_rows, int32_t* __restrict__ dst_tokens,
+              uint4* __restrict__ dst_rows, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
+    __shared__ int64_t src_row_of[MAX_TILE_ROWS];
+    const int S = (int)d_num[0];
+    const int64_t T = d_num[1];
+    if (T > capacity || S <= 0) return;      // capacity overflow was recorded by the scan kernel
+    const int64_t n_tiles = (T + tile_rows - 1) / tile_rows;
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int64_t t0 = tile * tile_rows;
+        const int rows_here = (int)min((int64_t)tile_rows, T - t0);
+        for (int r = threadIdx.x; r < rows_here; r += GATHER_THREADS) {
+            const int64_t t = t0 + r;
+            // largest s with cu_seqlens[s] <= t  (zero-length survivors are skipped by taking the last one)
+            int lo = 0, hi = S;                 // invariant: cu[lo] <= t < cu[hi]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+            }
+            const int64_t src = src_tok_off[survivor_idx[lo]] + (t - cu_seqlens[lo]);
+            src_row_of[r] = src;
+            if (dst_tokens) dst_tokens[t] = src_tokens[src];
+            if (tok_seq) tok_seq[t] = lo;
+            if (tok_adv) tok_adv[t] = adv[lo];
+        }
+        if (vec_per_row > 0) {
+            __syncthreads();
+            const int64_t total = (int64_t)rows_here * vec_per_row;
+            uint4* dst = dst_rows + t0 * vec_per_row;
+            int64_t v = threadIdx.x;
+            // eight 16-byte loads in flight per thread
+            for (; v + 7 * GATHER_THREADS < total; v += 8 * GATHER_THREADS) {
+                uint4 buf[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int64_t vv = v + u * GATHER_THREADS;
+                    const int r = (int)(vv / vec_per_row);
+                    const int c = (int)(vv - (int64_t)r * vec_per_row);
+                    buf[u] = ld_stream(src_rows + src_row_of[r] * vec_per_row + c);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) st_stream(dst + v + u * GATHER_THREADS, buf[u]);
+            }
+            for (; v < total; v += GATHER_THREADS) {
+                const int r = (int)(v / vec_per_row);
+                const int c = (int)(v - (int64_t)r * vec_per_row);
+                st_stream(dst + v, ld_stream(src_rows + src_row_of[r] * vec_per_row + c));
+            }
+            __syncthreads();
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths,
+                             const int64_t* src_tok_off, int32_t N, int32_t G, const int32_t* src_tokens,
+                             const void* src_rows, int32_t row_bytes, const float* rewards, float eps,
+                             int32_t ddof, int64_t dst_capacity_tokens, int32_t* dst_tokens, void* dst_rows,
+                             int64_t* cu_seqlens, int32_t* survivor_idx, float* adv, float* tok_adv,
+                             int32_t* tok_seq, int64_t* d_num, void* stream) {
+    if (!ctx || N < 0 || G < 1 || dst_capacity_tokens < 0 || ddof < 0 || !(eps >= 0.f)) return ARROL_ERR_INVALID_ARG;
+    if (!cu_seqlens || !d_num) return ARROL_ERR_INVALID_ARG;
+    if (N > 0 && (!keep || !lengths || !src_tok_off || !rewards || !survivor_idx || !adv))
+        return ARROL_ERR_INVALID_ARG;
+    if (N % G != 0) return ARROL_ERR_INVALID_ARG;
+    if ((src_tokens != nullptr) != (dst_tokens != nullptr)) return ARROL_ERR_INVALID_ARG;
+    if ((src_rows != nullptr) != (dst_rows != nullptr)) return ARROL_ERR_INVALID_ARG;
+    if (src_rows) {
+        if (row_bytes <= 0) return ARROL_ERR_INVALID_ARG;
+        if (row_bytes % 16 != 0) return ARROL_ERR_UNSUPPORTED;
+        if (!arrol_aligned(src_rows, 16) || !arrol_aligned(dst_rows, 16)) return ARROL_ERR_INVALID_ARG;
+    }
+    ArrolDeviceGuard guard(ctx->device);
+    if (!guard.ok) return ARROL_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    scan_adv_kernel<<<1, SCAN_THREADS, 0, s>>>(keep, lengths, N, G, rewards, (double)eps, ddof,
+                                               dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
+                                               ctx->d_status);
+    ARROL_CUDA_OK(cudaGetLastError());
+    const bool any_token_output = dst_tokens || dst_rows || tok_adv || tok_seq;
+    if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
+
+    const int vec_per_row = src_rows ? row_bytes / 16 : 0;
+    int tile_rows = MAX_TILE_ROWS;
+    if (vec_per_row > 0) {
+        // about 32 KB of payload per tile: eight 16-byte vectors per thread per pass
+        tile_rows = (8 * GATHER_THREADS) / vec_per_row;
+        if (tile_rows < 1) tile_rows = 1;
+        if (tile_rows > MAX_TILE_ROWS) tile_rows = MAX_TILE_ROWS;
+    }
+    const int64_t max_tiles = (dst_capacity_tokens + tile_rows - 1) / tile_rows;
+    int64_t blocks = (int64_t)ctx->sm_count * 8;
+    if (blocks > max_tiles) blocks = max_tiles;
+    if (blocks < 1) blocks = 1;
+    gather_kernel<<<(unsigned)blocks, GATHER_THREADS, 0, s>>>(
+        d_num, cu_seqlens, survivor_idx, src_tok_off, src_tokens, static_cast<const uint4*>(src_rows),
+        vec_per_row, adv, dst_capacity_tokens, tile_rows, dst_tokens, static_cast<uint4*>(dst_rows), tok_adv,
+        tok_seq);
+    ARROL_CUDA_OK(cudaGetLastError());
+    return ARROL_OK;
+}

@@ -1,0 +1,123 @@
+// Context life-cycle, status reporting and the host-side calibration-table helpers.
+#include <cmath>
+#include <new>
+
+#include "arrol_internal.h"
+
+extern "C" int arrol_version(void) { return 100; }
+
+extern "C" const char* arrol_status_string(int status) {
+    switch (status) {
+        case ARROL_OK: return "ok";
+        case ARROL_ERR_INVALID_ARG: return "invalid argument";
+        case ARROL_ERR_UNSUPPORTED: return "unsupported size or configuration";
+        case ARROL_ERR_WORKSPACE: return "workspace missing or too small";
+        case ARROL_ERR_CAPACITY: return "destination capacity exceeded (detected on the device)";
+        case ARROL_ERR_CUDA: return "a CUDA call failed";
+        case ARROL_ERR_DEVICE_STATUS: return "device-detected error (bad target id or expired wait)";
+        case ARROL_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int arrol_create(arrol_ctx** out, int device) {
+    if (!out) return ARROL_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count <= 0) {
+        (void)cudaGetLastError();
+        return ARROL_ERR_NO_DEVICE;
+    }
+    if (device < 0 || device >= count) return ARROL_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    ARROL_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return ARROL_ERR_NO_DEVICE;  // the kernels are built for sm_100a only
+    ArrolDeviceGuard guard(device);
+    if (!guard.ok) return ARROL_ERR_CUDA;
+
+    arrol_ctx* ctx = new (std::nothrow) arrol_ctx();
+    if (!ctx) return ARROL_ERR_CUDA;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->d_status = nullptr;
+    ctx->h_status = nullptr;
+    ctx->d_scratch = nullptr;
+    ctx->encode_tiled = nullptr;
+    bool ok = cudaMalloc(&ctx->d_status, 256) == cudaSuccess &&
+              cudaMemset(ctx->d_status, 0, 256) == cudaSuccess &&
+              cudaMallocHost(&ctx->h_status, 64) == cudaSuccess &&
+              cudaMalloc(&ctx->d_scratch, ARROL_SCRATCH_FLOATS * sizeof(float)) == cudaSuccess;
+    if (ok) {
+        cudaDriverEntryPointQueryResult qres;
+        void* fn = nullptr;
+        ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+             qres == cudaDriverEntryPointSuccess && fn != nullptr;
+        ctx->encode_tiled = fn;
+    }
+    if (!ok) {
+        (void)cudaGetLastError();
+        arrol_destroy(ctx);
+        return ARROL_ERR_CUDA;
+    }
+    *out = ctx;
+    return ARROL_OK;
+}
+
+extern "C" int arrol_destroy(arrol_ctx* ctx) {
+    if (!ctx) return ARROL_OK;
+    ArrolDeviceGuard guard(ctx->device);
+    if (ctx->d_status) (void)cudaFree(ctx->d_status);
+    if (ctx->h_status) (void)cudaFreeHost(ctx->h_status);
+    if (ctx->d_scratch) (void)cudaFree(ctx->d_scratch);
+    delete ctx;
+    return ARROL_OK;
+}
+
+extern "C" int arrol_poll_status(arrol_ctx* ctx, void* stream, uint32_t* dev_status_bits) {
+    if (!ctx) return ARROL_ERR_INVALID_ARG;
+    ArrolDeviceGuard guard(ctx->device);
+    if (!guard.ok) return ARROL_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    ARROL_CUDA_OK(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+    ARROL_CUDA_OK(cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), s));
+    ARROL_CUDA_OK(cudaStreamSynchronize(s));
+    uint32_t bits = *ctx->h_status;
+    if (dev_status_bits) *dev_status_bits = bits;
+    if (bits == 0) return ARROL_OK;
+    if (bits & (ARROL_DEV_BAD_TARGET | ARROL_DEV_WAIT_EXPIRED)) return ARROL_ERR_DEVICE_STATUS;
+    return ARROL_ERR_CAPACITY;
+}
+
+// ---- Binned posterior table (Appendix A.4), host side ----------------------------------------------
+
+extern "C" int arrol_calib_counts(const double* sprime, const uint8_t* y, int64_t n, int B, int64_t* cpos,
+                                  int64_t* cneg) {
+    if (B <= 0 || n < 0 || !cpos || !cneg || (n > 0 && (!sprime || !y))) return ARROL_ERR_INVALID_ARG;
+    for (int b = 0; b < B; ++b) { cpos[b] = 0; cneg[b] = 0; }
+    for (int64_t k = 0; k < n; ++k) {
+        double scaled = std::floor(sprime[k] * (double)B);
+        int b = scaled >= (double)(B - 1) ? B - 1 : (scaled <= 0.0 ? 0 : (int)scaled);
+        (y[k] ? cpos : cneg)[b] += 1;
+    }
+    return ARROL_OK;
+}
+
+extern "C" int arrol_build_q_lut(const int64_t* cpos, const int64_t* cneg, int B, double alpha, float* q_lut) {
+    if (B <= 0 || !cpos || !cneg || !q_lut || !(alpha >= 0.0)) return ARROL_ERR_INVALID_ARG;
+    double n_pos = 0.0, n_neg = 0.0;
+    for (int b = 0; b < B; ++b) {
+        if (cpos[b] < 0 || cneg[b] < 0) return ARROL_ERR_INVALID_ARG;
+        n_pos += (double)cpos[b];
+        n_neg += (double)cneg[b];
+    }
+    const double prior = (n_pos + n_neg) > 0.0 ? n_pos / (n_pos + n_neg) : 0.5;
+    const double den_pos = n_pos + alpha * B, den_neg = n_neg + alpha * B;
+    for (int b = 0; b < B; ++b) {
+        double like_pos = den_pos > 0.0 ? ((double)cpos[b] + alpha) / den_pos : 0.0;
+        double like_neg = den_neg > 0.0 ? ((double)cneg[b] + alpha) / den_neg : 0.0;
+        double num = prior * like_pos;
+        double den = num + (1.0 - prior) * like_neg;
+        q_lut[b] = den > 0.0 ? (float)(num / den) : (float)prior;  // an empty bin with alpha = 0 falls back to pi
+    }
+    return ARROL_OK;
+}

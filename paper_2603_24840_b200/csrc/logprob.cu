@@ -1,0 +1,482 @@
+// arrol_token_logprob: selected-token log-probability of every survivor token from the lm_head
+// (Section 3: log pi_theta(o_t | o_<t); Algorithm 1 "log-probs on R'"), as a fused contraction
+// hidden[T,d] x W_vocab[V,d]^T with an online max / log-sum-exp epilogue.  The T x V logits never leave the SM.
+//
+// One thread block per SM, persistent over work items (token tile of 128 rows, vocabulary split).  Per item the
+// block walks its vocabulary range in chunks of 256 columns.  Warp roles:
+//   warp 0      TMA producer: K-major, 128-byte-swizzled tiles of hidden (128 x 64) and W_vocab (256 x 64) into
+//               a ring of shared-memory stages, completion on mbarriers
+//   warp 1      tcgen05.mma issuer (one elected lane): 128 x 256 x 16 bf16 MMAs into one of two 256-column fp32
+//               accumulators in tensor memory; tcgen05.commit releases stages / publishes accumulators
+//   warps 2..5  epilogue: thread r owns token row r of the tile; tcgen05.ld of its accumulator row, running
+//               maximum and sum of 2^(z log2e - max), and the target column's logit, all in registers
+// The two accumulators let the epilogue of chunk c overlap the MMAs of chunk c + 1.
+// Every wait is bounded; when one runs out the block records ARROL_DEV_WAIT_EXPIRED, drains and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "arrol_internal.h"
+
+namespace {
+
+constexpr int BM = 128;          // token rows per tile  (MMA M)
+constexpr int BN = 256;          // vocabulary columns per chunk (MMA N)
+constexpr int BK = 64;           // bf16 elements per stage along d: 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;       // K of one tcgen05.mma for 16-bit inputs
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
+constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KB
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int TMEM_COLS = 512;   // two fp32 accumulators of BN columns
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_THREADS = 128;
+constexpr uint32_t SPIN_LIMIT = 1u << 26;    // tries per wait before giving up (each try can suspend ~us)
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+
+struct PartialLse {   // per (split, token): running maximum and sum in the base-2 domain, target logit
+    float m2, l, zy2, pad;
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1u;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_alloc(uint32_t* smem_result, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+                 "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void tcgen05_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives lane (base + i), columns c .. c+31
+__device__ __forceinline__ void tcgen05_ld_32x32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with the 128-byte
+// swizzle: 8-row groups are 1024 bytes apart (stride byte offset); the leading byte offset is unused for this
+// layout.  Bits: [0,14) address >> 4, [16,30) LBO >> 4, [32,46) SBO >> 4, [46,48) = 1, [61,64) = 2 (128B swizzle).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+    uint64_t desc = 0;
+    desc |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    desc |= (uint64_t)1 << 16;
+    desc |= (uint64_t)(1024 >> 4) << 32;
+    desc |= (uint64_t)1 << 46;
+    desc |= (uint64_t)2 << 61;
+    return desc;
+}
+// Instruction descriptor, kind::f16: D = f32 (bits 4-5 = 1), A = B = bf16 (bits 7-9, 10-12 = 1), both K-major,
+// N >> 3 at bits 17-22, M >> 4 at bits 24-28.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct LogprobParams {
+    const int32_t* targets;
+    const int64_t* d_T;
+    int64_t T_max;
+    int d, V;
+    int splits;            // vocabulary splits per token tile
+    int chunks_per_split;  // chunks of BN columns per split
+    float scale2;          // inv_temperature * log2(e)
+    float* logp;
+    float* lse;
+    PartialLse* partial;   // [splits][T_max] when splits > 1
+    uint32_t* d_status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
+                     const LogprobParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* stage_a = smem;
+    uint8_t* stage_b = smem + (size_t)STAGES * A_STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t* full = bars;                    // [STAGES]  TMA -> MMA
+    uint64_t* empty = bars + STAGES;          // [STAGES]  MMA -> TMA
+    uint64_t* acc_full = bars + 2 * STAGES;   // [2]       MMA -> epilogue
+    uint64_t* acc_empty = acc_full + 2;       // [2]       epilogue -> MMA
+    uint64_t* drain = acc_empty + 2;          // [1]       used only when giving up: MMAs in flight -> done
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    int64_t T = p.T_max;
+    if (p.d_T) { const int64_t t = *p.d_T; T = t < 0 ? 0 : (t < T ? t : T); }
+    const int64_t m_tiles = (T + BM - 1) / BM;
+    const int64_t items = m_tiles * p.splits;
+    const int k_steps = (p.d + BK - 1) / BK;
+    const int total_chunks = (p.V + BN - 1) / BN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_THREADS / 32); }
+        mbar_init(drain, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_h) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+    }
+    if (warp == 1) {
+        tcgen05_alloc(tmem_slot, TMEM_COLS);
+        tcgen05_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+                const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
+                const int c0 = split * p.chunks_per_split;
+                const int c1 = min(c0 + p.chunks_per_split, total_chunks);
+                for (int c = c0; c < c1 && ok; ++c) {
+                    for (int ks = 0; ks < k_steps; ++ks) {
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                        mbar_expect_tx(&full[stage], STAGE_BYTES);
+                        tma_load_2d(stage_a + (size_t)stage * A_STAGE_BYTES, &map_h, ks * BK, m_tile * BM, &full[stage]);
+                        tma_load_2d(stage_b + (size_t)stage * B_STAGE_BYTES, &map_w, ks * BK, c * BN, &full[stage]);
+                        ++issued;
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                // Gave up: let the copies already issued land before the block's shared memory goes away.
+                // The last min(issued, STAGES) stages may still be in flight; wait for each (bounded).
+                const uint32_t pending = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
+                uint32_t s = stage, ph = phase;
+                for (uint32_t i = 0; i < pending; ++i) {
+                    if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+                    for (uint32_t it = 0; it < SPIN_LIMIT; ++it)
+                        if (mbar_try_wait(&full[s], ph)) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BM, BN);
+            uint32_t stage = 0, phase = 0;
+            uint32_t acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+                const int split = (int)(item % p.splits);
+                const int c0 = split * p.chunks_per_split;
+                const int c1 = min(c0 + p.chunks_per_split, total_chunks);
+                for (int c = c0; c < c1 && ok; ++c) {
+                    if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * BN;
+                    for (int ks = 0; ks < k_steps; ++ks) {
+                        if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+                        tcgen05_fence_after();
+                        const uint64_t a_desc = make_smem_desc(smem_u32(stage_a + (size_t)stage * A_STAGE_BYTES));
+                        const uint64_t b_desc = make_smem_desc(smem_u32(stage_b + (size_t)stage * B_STAGE_BYTES));
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k) {
+                            // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in address units
+                            tcgen05_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                             (ks | k) != 0 ? 1u : 0u);
+                        }
+                        tcgen05_commit(&empty[stage]);   // stage reusable once these MMAs have read it
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (ok) tcgen05_commit(&acc_full[acc]);   // accumulator complete
+                    if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // Gave up: wait (bounded) until the MMAs already issued have finished with shared and tensor memory.
+                tcgen05_commit(drain);
+                for (uint32_t it = 0; it < SPIN_LIMIT; ++it)
+                    if (mbar_try_wait(drain, 0u)) break;
+            }
+        }
+    } else {
+        // ---------------- epilogue: one token row per thread ----------------
+        const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. 32*quarter+31
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
+            const int c0 = split * p.chunks_per_split;
+            const int c1 = min(c0 + p.chunks_per_split, total_chunks);
+            const int64_t t = (int64_t)m_tile * BM + row_in_tile;
+            const int y = (t < T) ? p.targets[t] : -1;
+            float m2 = -INFINITY, l = 0.f, zy2 = -INFINITY;
+            for (int c = c0; c < c1 && ok; ++c) {
+                ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
+                ok = __all_sync(0xffffffffu, ok) != 0;     // keep the warp converged for the aligned tensor-memory loads
+                if (!ok) break;
+                tcgen05_fence_after();
+                const int col0 = c * BN;
+#pragma unroll 1
+                for (int piece = 0; piece < BN / 32; ++piece) {
+                    const int pc0 = col0 + piece * 32;
+                    if (pc0 >= p.V) break;                  // columns past the vocabulary (zero-filled by TMA)
+                    float v[32];
+                    tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
+                    if (pc0 + 32 > p.V) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) if (pc0 + j >= p.V) v[j] = -INFINITY;
+                    }
+                    if ((unsigned)(y - pc0) < 32u) {
+                        const int jy = y - pc0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) if (j == jy) zy2 = v[j] * p.scale2;
+                    }
+                    float bmax = v[0];
+#pragma unroll
+                    for (int j = 1; j < 32; ++j) bmax = fmaxf(bmax, v[j]);
+                    const float m_new = fmaxf(m2, bmax * p.scale2);
+                    float sum = 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) sum += ex2_approx(fmaf(v[j], p.scale2, -m_new));
+                    l = fmaf(l, ex2_approx(m2 - m_new), sum);
+                    m2 = m_new;
+                }
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&acc_empty[acc]);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            if (ok && t < T) {
+                if (p.splits == 1) {
+                    const float lse2 = m2 + log2f(l);
+                    const float ln2 = 0.69314718055994530942f;
+                    float out = 0.f;
+                    if (y >= 0) {
+                        if (y < p.V) out = (zy2 - lse2) * ln2;
+                        else atomicOr(p.d_status, ARROL_DEV_BAD_TARGET);
+                    }
+                    p.logp[t] = out;
+                    if (p.lse) p.lse[t] = lse2 * ln2;
+                } else {
+                    PartialLse pr;
+                    pr.m2 = m2; pr.l = l; pr.zy2 = zy2; pr.pad = 0.f;
+                    *reinterpret_cast<float4*>(&p.partial[(int64_t)split * p.T_max + t]) =
+                        make_float4(pr.m2, pr.l, pr.zy2, pr.pad);
+                }
+            }
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.d_status, ARROL_DEV_WAIT_EXPIRED);
+    if (warp == 1) {
+        tcgen05_fence_after();
+        tcgen05_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// Merge of the per-split (max, sum, target logit) triples: M = max m_s, L = sum l_s 2^(m_s - M).
+__global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, const int32_t* __restrict__ targets,
+                                      const int64_t* __restrict__ d_T, int64_t T_max, int V, int splits,
+                                      float* __restrict__ logp, float* __restrict__ lse, uint32_t* d_status) {
+    int64_t T = T_max;
+    if (d_T) { const int64_t t = *d_T; T = t < 0 ? 0 : (t < T ? t : T); }
+    for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
+        float M = -INFINITY, zy2 = -INFINITY;
+        for (int s = 0; s < splits; ++s) {
+            const float4 pr = *reinterpret_cast<const float4*>(&partial[(int64_t)s * T_max + t]);
+            M = fmaxf(M, pr.x);
+            zy2 = fmaxf(zy2, pr.z);          // exactly one split holds the target column; the others hold -inf
+        }
+        float L = 0.f;
+        for (int s = 0; s < splits; ++s) {
+            const float4 pr = *reinterpret_cast<const float4*>(&partial[(int64_t)s * T_max + t]);
+            L += pr.y * exp2f(pr.x - M);
+        }
+        const float lse2 = M + log2f(L);
+        const float ln2 = 0.69314718055994530942f;
+        const int y = targets[t];
+        float out = 0.f;
+        if (y >= 0) {
+            if (y < V) out = (zy2 - lse2) * ln2;
+            else atomicOr(d_status, ARROL_DEV_BAD_TARGET);
+        }
+        logp[t] = out;
+        if (lse) lse[t] = lse2 * ln2;
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// [rows, cols] bf16 row-major -> tiles of box_rows x 64 columns, 128-byte swizzle, zero fill outside
+int make_map(arrol_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? ARROL_OK : ARROL_ERR_CUDA;
+}
+
+// How many vocabulary splits per token tile.  With one split every resident block streams a different token
+// tile (128 x d x 2 bytes each) against the same W chunks; when those tiles together outgrow about half of L2
+// the tiles would be re-fetched from HBM once per chunk, so the vocabulary is split until they fit.
+int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
+    const int total_chunks = (V + BN - 1) / BN;
+    const int64_t m_tiles = (T_max + BM - 1) / BM;
+    int splits = 1;
+    const double l2_budget = 48.0 * 1024 * 1024;
+    const double tile_bytes = (double)BM * d * 2;
+    while (splits < 8 && (ctx->sm_count / splits) * tile_bytes > l2_budget) splits *= 2;
+    // few token tiles: split so that every SM has work
+    while (splits < 16 && m_tiles * splits < ctx->sm_count && splits * 2 <= total_chunks) splits *= 2;
+    if (splits > total_chunks) splits = total_chunks;
+    return splits < 1 ? 1 : splits;
+}
+
+}  // namespace
+
+extern "C" size_t arrol_token_logprob_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
+    if (!ctx || T_max <= 0 || d <= 0 || V <= 0) return 0;
+    const int splits = choose_splits(ctx, T_max, d, V);
+    if (splits <= 1) return 256;   // never zero, so that callers can always pass a valid pointer
+    return (size_t)splits * (size_t)T_max * sizeof(PartialLse) + 256;
+}
+
+extern "C" int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                                   int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
+                                   float* logp, float* lse, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+    if (!ctx || T_max < 0 || d <= 0 || V <= 0 || !(inv_temperature > 0.f)) return ARROL_ERR_INVALID_ARG;
+    if (T_max == 0) return ARROL_OK;
+    if (!hidden || !W_vocab || !targets || !logp) return ARROL_ERR_INVALID_ARG;
+    if (d % 8 != 0) return ARROL_ERR_UNSUPPORTED;
+    if (!arrol_aligned(hidden, 16) || !arrol_aligned(W_vocab, 16)) return ARROL_ERR_INVALID_ARG;
+    if (T_max > (int64_t)INT32_MAX - BM) return ARROL_ERR_UNSUPPORTED;   // TMA coordinates are 32-bit
+    const size_t need = arrol_token_logprob_workspace(ctx, T_max, d, V);
+    if (!workspace || workspace_bytes < need || !arrol_aligned(workspace, 256)) return ARROL_ERR_WORKSPACE;
+
+    ArrolDeviceGuard guard(ctx->device);
+    if (!guard.ok) return ARROL_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+
+    CUtensorMap map_h, map_w;
+    if (make_map(ctx, &map_h, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+
+    LogprobParams p;
+    p.targets = targets;
+    p.d_T = d_T;
+    p.T_max = T_max;
+    p.d = d;
+    p.V = V;
+    p.splits = choose_splits(ctx, T_max, d, V);
+    const int total_chunks = (V + BN - 1) / BN;
+    p.chunks_per_split = (total_chunks + p.splits - 1) / p.splits;
+    p.splits = (total_chunks + p.chunks_per_split - 1) / p.chunks_per_split;   // no empty split
+    p.scale2 = inv_temperature * 1.44269504088896340736f;
+    p.logp = logp;
+    p.lse = lse;
+    p.partial = static_cast<PartialLse*>(workspace);
+    p.d_status = ctx->d_status;
+
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES));
+    const int64_t m_tiles = (T_max + BM - 1) / BM;
+    int64_t grid = m_tiles * p.splits;
+    if (grid > ctx->sm_count) grid = ctx->sm_count;
+    token_logprob_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
+    ARROL_CUDA_OK(cudaGetLastError());
+    if (p.splits > 1) {
+        int64_t blocks = (T_max + 255) / 256;
+        if (blocks > (int64_t)ctx->sm_count * 8) blocks = (int64_t)ctx->sm_count * 8;
+        combine_splits_kernel<<<(unsigned)blocks, 256, 0, s>>>(p.partial, targets, d_T, T_max, V, p.splits, logp,
+                                                              lse, ctx->d_status);
+        ARROL_CUDA_OK(cudaGetLastError());
+    }
+    return ARROL_OK;
+}
