@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the prune-and-rebatch hot path on B200.
+
+A step is one pass of the whole path over one batch of synthetic input shaped like a GRPO/DAPO run:
+  arrol_score_partial -> arrol_select -> arrol_compact (token ids + hidden rows) -> arrol_token_logprob.
+`value` = survivor tokens processed per second over the whole step, inputs resident in HBM.
+`e2e`   = the same metric through arrol_prune_rebatch_host: inputs in pinned host memory, results read back.
+`--impl reference` times the CPU oracle (the plain fp64 program the GPU path is checked against) on host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "survivor_logprob_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM traffic of one token_logprob launch per survivor token, from the ncu capture summarised under profiles/
+# (bytes read + written divided by the tokens of the captured launch); None until a capture exists.
+LOGPROB_DRAM_BYTES_PER_TOKEN = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
+        return {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and the --impl reference arm)
+# ------------------------------------------------------------------------------------------------------------
+def oracle_step_rate(w, budget_s: float, logp_rows=None):
+    """Times the oracle on the workload: head scoring, probability map, selection, scan, token gather and
+    advantages at full size; the fp64 log-softmax gather on a bounded sample of survivor tokens.  Returns
+    (tokens_per_s for the whole path, description, cores, seconds spent)."""
+    import torch
+    import oracle
+    from paper_2603_24840_b200 import synth
+
+    t_begin = time.perf_counter()
+    ell = synth.lengths(w)
+    off = synth.src_offsets(ell)
+    rew = synth.rewards(w)
+    head = synth.head_weights(w)
+    tokens = synth.token_ids(w, int(off[-1]))
+    hist_s, hist_y = synth.calib_history(w)
+    oa = lambda t: None if t is None else synth.as_oracle_array(t)
+    x_cut = synth.hidden_states(w, w.N, stream=21)           # hidden rows at the detection length
+    Wv = oa(synth.vocab_weights(w, dtype=torch.bfloat16))
+    cores = oracle.num_threads()
+
+    t0 = time.perf_counter()
+    s = oracle.head_score(oa(x_cut), oa(head["W1"]), oa(head["b1"]), oa(head["w2"]), oa(head["b2"]), h=w.h)
+    _, lut = oracle.build_q_lut(*oracle.calib_counts(hist_s, hist_y, w.B), 1.0)
+    _, _, q = oracle.prob_map(s, lut)
+    keep = oracle.select(q.astype(np.float32), w.P, w.G, w.K, w.rho)
+    idx, cu, S, T = oracle.survivor_scan(keep, ell)
+    dst_tokens, _, _ = oracle.gather(idx, cu, off[:-1], tokens)
+    oracle.advantages(rew, keep, w.G)
+    t_prune = time.perf_counter() - t0
+
+    # log-prob sample: calibrate on one row per core, then size the sample to the budget
+    probe = max(cores, 1)
+    H = oa(synth.hidden_states(w, max(probe, 1), stream=22).to(torch.bfloat16))
+    t0 = time.perf_counter()
+    oracle.token_logprob(H, Wv, dst_tokens[:probe])
+    t_probe = time.perf_counter() - t0
+    per_row = t_probe / probe
+    n = int(max(probe, min(T, (budget_s - t_probe) / max(per_row, 1e-9))))
+    if logp_rows is not None:
+        n = min(n, logp_rows)
+    n = max(probe, (n // probe) * probe)
+    H = oa(synth.hidden_states(w, n, stream=23).to(torch.bfloat16))
+    t0 = time.perf_counter()
+    oracle.token_logprob(H, Wv, dst_tokens[:n])
+    t_logp = time.perf_counter() - t0
+    per_tok = t_logp / n
+    tokens_per_s = T / (t_prune + per_tok * T)
+    sample = ("scoring/selection/scan/token-gather/advantages at full size (%.3f s); fp64 log-softmax gather on %d of "
+              "%d survivor tokens (%.1f s), extrapolated per token" % (t_prune, n, T, t_logp))
+    return tokens_per_s, sample, cores, time.perf_counter() - t_begin
+
+
+def run_reference(args, w):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    vals = []
+    budget = max(2.0, min(30.0, 120.0 / max(1, args.steps + args.warmup)))
+    sample = ""
+    cores = 0
+    for i in range(args.warmup + args.steps):
+        v, sample, cores, _ = oracle_step_rate(w, budget)
+        if i >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    ell_T = value
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": None, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "CPU oracle on host cores; each step a bounded sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    del ell_T
+    print(json.dumps(out), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2603_24840_b200 import binding as B
+    from paper_2603_24840_b200 import synth
+    from paper_2603_24840_b200.pipeline import PruneRebatch, host_inputs
+    import dataclasses
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    # weak scaling: every rank prunes and re-batches its own prompts (different seed per rank), no exchange
+    w_rank = dataclasses.replace(w, seed=w.seed + 1000 * rank)
+
+    pr = PruneRebatch(w_rank, device=local, with_rows=True)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        pr.step()
+    barrier()
+    S, T = pr.counts()
+    B.arrol_poll_status(pr.ctx)
+
+    # ---- timed region: device-resident inputs ----
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
+    sampler = ClockSampler(local)
+    launches0 = B.arrol_launch_count(pr.ctx)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for k in range(K):
+        ev[k][0].record(stream)
+        pr.score_partial()
+        ev[k][1].record(stream)
+        pr.select()
+        ev[k][2].record(stream)
+        pr.compact()
+        ev[k][3].record(stream)
+        pr.token_logprob()
+        ev[k][4].record(stream)
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    launches = B.arrol_launch_count(pr.ctx) - launches0
+    total_ms = t_start.elapsed_time(t_end)
+    B.arrol_poll_status(pr.ctx)
+    seg = np.array([[ev[k][i].elapsed_time(ev[k][i + 1]) for i in range(4)] for k in range(K)])  # ms
+    seg_mean = seg.mean(0)
+
+    # prune step without the hidden-row plane (token ids only), timed separately
+    for _ in range(2):
+        pr.prune_step(with_rows=False)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(K):
+        pr.prune_step(with_rows=False)
+    b.record(stream)
+    torch.cuda.synchronize()
+    prune_tokens_only_us = a.elapsed_time(b) / K * 1e3
+
+    # ---- e2e: host buffers through arrol_prune_rebatch_host ----
+    e2e = run_e2e(args, w_rank, pr, B, torch, world, barrier)
+
+    # ---- reduce over ranks ----
+    t_total = torch.tensor([total_ms, e2e["ms_per_step"]], dtype=torch.float64, device="cuda")
+    tok = torch.tensor([float(T)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_total, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
+    total_ms_max = float(t_total[0])
+    e2e_ms_max = float(t_total[1])
+    tokens_all = float(tok[0])
+
+    if rank == 0:
+        peaks = load_peaks()
+        ms_per_step = total_ms_max / K
+        value = tokens_all / (ms_per_step * 1e-3)
+        logp_ms = float(seg_mean[3])
+        flops = 2.0 * T * w.d * w.V
+        achieved = flops / (logp_ms * 1e-3) / 1e12
+        peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+        gather_bytes = 2.0 * T * w.d * 2 + 8.0 * T
+        roofline = {
+            "kernel": "token_logprob_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
+            "unit": "TFLOP/s", "frac": achieved / peak,
+            "peak_source": "%s bf16 sustained (kernel timed inside a long step)" % peaks["source"],
+            "frac_of_burst": achieved / float(peaks["bf16_tflops"]), "frac_of_nominal_2250": achieved / 2250.0,
+            "traffic": None if LOGPROB_DRAM_BYTES_PER_TOKEN is None else LOGPROB_DRAM_BYTES_PER_TOKEN * T,
+            "algorithmic_flops_per_launch": flops,
+            "launch_ms": logp_ms,
+        }
+        compact_gbs = gather_bytes / (float(seg_mean[2]) * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "P": w.P, "G": w.G, "K": w.K, "cutoff": w.cutoff, "d": w.d, "V": w.V,
+                       "head_h": w.h, "survivors": S, "survivor_tokens": T, "source_rows": pr.T_src,
+                       "l2": "inputs larger than L2 (hidden rows %.2f GB, W_vocab %.2f GB)" % (
+                           pr.T_src * w.d * 2 / 1e9, w.V * w.d * 2 / 1e9)},
+            "clocks": clocks,
+            "e2e": {"value": tokens_all / (e2e_ms_max * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                    "ms_per_step": e2e_ms_max},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "breakdown_ms": {"score_partial": float(seg_mean[0]), "select": float(seg_mean[1]),
+                             "compact": float(seg_mean[2]), "token_logprob": logp_ms},
+            "logprob_tokens_per_s": T / (logp_ms * 1e-3),
+            "prune_step_us": {"tokens_only": prune_tokens_only_us,
+                              "with_hidden_rows": float(seg_mean[:3].sum()) * 1e3},
+            "compact_roofline": {"bound": "hbm", "achieved": compact_gbs, "peak": float(peaks["hbm_gbs"]),
+                                 "unit": "GB/s", "frac": compact_gbs / float(peaks["hbm_gbs"]),
+                                 "algorithmic_bytes_per_launch": gather_bytes},
+        }
+        if not args.no_cpu_baseline and world == 1:
+            v, sample, cores, _ = oracle_step_rate(w, args.cpu_budget)
+            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        else:
+            out["cpu_baseline"] = None
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, w, pr, B, torch, world, barrier):
+    """Same step through the host-buffer entry point: every step copies the inputs from pinned host memory and
+    reads the results back."""
+    N, cap, d = w.N, pr.cap, w.d
+    pin = lambda t: t.cpu().pin_memory()
+    h = {
+        "h_hidden": pin(pr.src_rows), "h_src_tokens": pin(pr.src_tokens), "h_lengths": pin(pr.lengths),
+        "h_src_tok_off": pin(pr.src_tok_off), "h_rewards": pin(pr.rewards),
+        "h_logp": torch.empty(cap, dtype=torch.float32).pin_memory(),
+        "h_adv": torch.empty(N, dtype=torch.float32).pin_memory(),
+        "h_cu_seqlens": torch.empty(N + 1, dtype=torch.int64).pin_memory(),
+        "h_survivor_idx": torch.empty(N, dtype=torch.int32).pin_memory(),
+        "h_num": torch.empty(2, dtype=torch.int64).pin_memory(),
+    }
+    dv = {
+        "W_vocab": pr.W_vocab, "d_hidden": torch.empty_like(pr.src_rows), "d_src_tokens": torch.empty_like(pr.src_tokens),
+        "d_lengths": torch.empty_like(pr.lengths), "d_src_tok_off": torch.empty_like(pr.src_tok_off),
+        "d_row_index": torch.empty_like(pr.row_index), "d_rewards": torch.empty_like(pr.rewards),
+        "d_score": pr.score, "d_prob": pr.prob, "d_q": pr.q, "d_keep": pr.keep, "d_survivor_idx": pr.survivor_idx,
+        "d_cu_seqlens": pr.cu_seqlens, "d_adv": pr.adv, "d_num": pr.d_num, "d_dst_tokens": pr.dst_tokens,
+        "d_dst_rows": pr.dst_rows, "d_logp": pr.logp, "d_workspace": pr.workspace,
+    }
+    scal = dict(P=w.P, G=w.G, K=w.K, cutoff=w.cutoff, d=w.d, V=w.V, ddof=0, rho=w.rho, eps=1e-6,
+                inv_temperature=1.0, T_src=pr.T_src, dst_capacity_tokens=cap)
+    head = dict(pr.head)
+    if pr.hidden_score.dtype != torch.bfloat16:   # fp32 workload: the host-step entry takes bf16 state
+        head = {k: (v.to(torch.bfloat16) if torch.is_tensor(v) else v) for k, v in head.items()}
+    tensors = dict(h)
+    tensors.update(dv)
+    step = B.make_host_step(scal, head, pr.q_lut, tensors)
+    h2d = sum(h[k].numel() * h[k].element_size() for k in ("h_hidden", "h_src_tokens", "h_lengths", "h_src_tok_off",
+                                                           "h_rewards"))
+    d2h = sum(h[k].numel() * h[k].element_size() for k in ("h_logp", "h_adv", "h_cu_seqlens", "h_survivor_idx", "h_num"))
+    n_e2e = max(1, min(args.steps, 5))
+    for _ in range(2):
+        B.arrol_prune_rebatch_host(pr.ctx, step)
+    barrier()
+    stream = torch.cuda.current_stream()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(n_e2e):
+        B.arrol_prune_rebatch_host(pr.ctx, step)       # synchronous: returns with results in host memory
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / n_e2e
+    assert int(h["h_num"][1]) == pr.counts()[1]
+    return {"ms_per_step": ms, "h2d": int(h2d), "d2h": int(d2h)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama-3.2-1b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
+    args = ap.parse_args()
+    from paper_2603_24840_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

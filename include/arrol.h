@@ -149,6 +149,64 @@ int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab,
                         int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                         float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- Whole step from host buffers (Algorithm 1, frontend lines "filter ... rebatch ... log-probs on R'") --
+ * Convenience call for callers whose per-step data lives in host memory: copies the step's inputs to the device
+ * staging buffers, runs arrol_score_partial -> arrol_select -> arrol_compact -> arrol_token_logprob on `stream`,
+ * copies the results back and waits for the stream.  Synchronous; allocates nothing.
+ * The quality head reads, for rollout i, source row src_tok_off[i] + cutoff - 1 (its hidden state at the
+ * detection length); the same source rows are the payload that is compacted and fed to the lm_head.
+ * Pointers prefixed h_ are HOST pointers (pinned memory gives full copy speed), d_ are DEVICE buffers provided by
+ * the caller with at least the stated sizes.  Model state (head, calib, W_vocab) is device-resident. */
+typedef struct arrol_host_step {
+    int32_t P, G, K, cutoff;       /* prompts, group size, survivors per group, detection length (>= 1)         */
+    int32_t d, V;                  /* hidden width, vocabulary                                                  */
+    int32_t ddof, reserved;
+    double rho;                    /* target positive ratio                                                     */
+    float eps, inv_temperature;
+    int64_t T_src;                 /* source rows (sum of stored rollout lengths)                               */
+    int64_t dst_capacity_tokens;   /* capacity of the packed buffers, in tokens                                 */
+    /* inputs, host */
+    const void* h_hidden;          /* [T_src, d] bf16                                                           */
+    const int32_t* h_src_tokens;   /* [T_src]                                                                   */
+    const int32_t* h_lengths;      /* [P*G]                                                                     */
+    const int64_t* h_src_tok_off;  /* [P*G]                                                                     */
+    const float* h_rewards;        /* [P*G]                                                                     */
+    /* model state, device */
+    arrol_head head;               /* dtype must be ARROL_BF16                                                  */
+    arrol_calib calib;
+    const void* W_vocab;           /* [V, d] bf16                                                               */
+    /* staging and outputs, device */
+    void* d_hidden;                /* [T_src, d] bf16                                                           */
+    int32_t* d_src_tokens;         /* [T_src]                                                                   */
+    int32_t* d_lengths;            /* [P*G]                                                                     */
+    int64_t* d_src_tok_off;        /* [P*G]                                                                     */
+    int64_t* d_row_index;          /* [P*G]                                                                     */
+    float* d_rewards;              /* [P*G]                                                                     */
+    float *d_score, *d_prob, *d_q; /* [P*G] each                                                                */
+    uint8_t* d_keep;               /* [P*G]                                                                     */
+    int32_t* d_survivor_idx;       /* [P*G]                                                                     */
+    int64_t* d_cu_seqlens;         /* [P*G + 1]                                                                 */
+    float* d_adv;                  /* [P*G]                                                                     */
+    int64_t* d_num;                /* [2]                                                                       */
+    int32_t* d_dst_tokens;         /* [cap]                                                                     */
+    void* d_dst_rows;              /* [cap, d] bf16                                                             */
+    float* d_logp;                 /* [cap]                                                                     */
+    void* d_workspace;             /* arrol_token_logprob_workspace(ctx, cap, d, V) bytes, 256-byte aligned     */
+    size_t workspace_bytes;
+    /* results, host */
+    float* h_logp;                 /* [cap]; entries >= T are not meaningful                                    */
+    float* h_adv;                  /* [P*G]; first S entries                                                    */
+    int64_t* h_cu_seqlens;         /* [P*G + 1]; first S + 1 entries                                            */
+    int32_t* h_survivor_idx;       /* [P*G]; first S entries                                                    */
+    int64_t* h_num;                /* [2] = {S, T}                                                              */
+} arrol_host_step;
+
+/* Returns ARROL_OK, a validation/launch error, or the device status translated as by arrol_poll_status. */
+int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* step, void* stream);
+
+/* Number of kernels this context has launched so far (host-side count; -1 for a NULL context). */
+int64_t arrol_launch_count(arrol_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

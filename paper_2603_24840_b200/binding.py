@@ -20,7 +20,7 @@ DEV_CAPACITY, DEV_BAD_TARGET, DEV_WAIT_EXPIRED = 1, 2, 4
 EXPORTS = [
     "arrol_version", "arrol_status_string", "arrol_create", "arrol_destroy", "arrol_poll_status",
     "arrol_calib_counts", "arrol_build_q_lut", "arrol_score_partial", "arrol_select", "arrol_compact",
-    "arrol_token_logprob_workspace", "arrol_token_logprob",
+    "arrol_token_logprob_workspace", "arrol_token_logprob", "arrol_prune_rebatch_host", "arrol_launch_count",
 ]
 
 
@@ -37,6 +37,24 @@ class _Head(C.Structure):
 
 class _Calib(C.Structure):
     _fields_ = [("B", C.c_int32), ("reserved", C.c_int32), ("q_lut", C.c_void_p)]
+
+
+class _HostStep(C.Structure):
+    _fields_ = [("P", C.c_int32), ("G", C.c_int32), ("K", C.c_int32), ("cutoff", C.c_int32),
+                ("d", C.c_int32), ("V", C.c_int32), ("ddof", C.c_int32), ("reserved", C.c_int32),
+                ("rho", C.c_double), ("eps", C.c_float), ("inv_temperature", C.c_float),
+                ("T_src", C.c_int64), ("dst_capacity_tokens", C.c_int64),
+                ("h_hidden", C.c_void_p), ("h_src_tokens", C.c_void_p), ("h_lengths", C.c_void_p),
+                ("h_src_tok_off", C.c_void_p), ("h_rewards", C.c_void_p),
+                ("head", _Head), ("calib", _Calib), ("W_vocab", C.c_void_p),
+                ("d_hidden", C.c_void_p), ("d_src_tokens", C.c_void_p), ("d_lengths", C.c_void_p),
+                ("d_src_tok_off", C.c_void_p), ("d_row_index", C.c_void_p), ("d_rewards", C.c_void_p),
+                ("d_score", C.c_void_p), ("d_prob", C.c_void_p), ("d_q", C.c_void_p), ("d_keep", C.c_void_p),
+                ("d_survivor_idx", C.c_void_p), ("d_cu_seqlens", C.c_void_p), ("d_adv", C.c_void_p),
+                ("d_num", C.c_void_p), ("d_dst_tokens", C.c_void_p), ("d_dst_rows", C.c_void_p),
+                ("d_logp", C.c_void_p), ("d_workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("h_logp", C.c_void_p), ("h_adv", C.c_void_p), ("h_cu_seqlens", C.c_void_p),
+                ("h_survivor_idx", C.c_void_p), ("h_num", C.c_void_p)]
 
 
 _lib = None
@@ -73,6 +91,10 @@ def load_library():
     lib.arrol_token_logprob.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                         C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_size_t, C.c_void_p]
+    lib.arrol_prune_rebatch_host.argtypes = [C.c_void_p, C.POINTER(_HostStep), C.c_void_p]
+    lib.arrol_prune_rebatch_host.restype = C.c_int
+    lib.arrol_launch_count.argtypes = [C.c_void_p]
+    lib.arrol_launch_count.restype = C.c_int64
     for fn in ("arrol_create", "arrol_destroy", "arrol_poll_status", "arrol_calib_counts", "arrol_build_q_lut",
                "arrol_score_partial", "arrol_select", "arrol_compact", "arrol_token_logprob"):
         getattr(lib, fn).restype = C.c_int
@@ -219,3 +241,41 @@ def arrol_token_logprob(ctx: Context, hidden, W_vocab, targets, T_max: int, d: i
                                               _ptr(lse), _ptr(workspace),
                                               0 if workspace is None else workspace.numel() * workspace.element_size(),
                                               _stream(stream)), "arrol_token_logprob")
+
+
+def arrol_launch_count(ctx: Context) -> int:
+    return int(load_library().arrol_launch_count(ctx.handle))
+
+
+def _fill_head(hs: _Head, hidden_dtype_code: int, d: int, head: dict):
+    hs.d = int(d)
+    hs.h = int(head.get("h", 0))
+    hs.dtype = hidden_dtype_code
+    for name in ("W1", "b1", "w2", "b2"):
+        t = head.get(name)
+        setattr(hs, name, None if t is None else t.data_ptr())
+
+
+def make_host_step(scalars: dict, head: dict, q_lut: Optional[torch.Tensor], tensors: dict) -> _HostStep:
+    """Builds the argument block of arrol_prune_rebatch_host.  `scalars`: P, G, K, cutoff, d, V, rho, eps, ddof,
+    inv_temperature, T_src, dst_capacity_tokens.  `tensors`: every h_* (CPU tensors) and d_* (CUDA tensors) field
+    plus W_vocab.  The caller keeps the tensors alive while the block is in use."""
+    st = _HostStep()
+    for k, v in scalars.items():
+        setattr(st, k, v)
+    _fill_head(st.head, ARROL_BF16, scalars["d"], head)
+    st.calib.B = 0 if q_lut is None else q_lut.shape[0]
+    st.calib.q_lut = None if q_lut is None else q_lut.data_ptr()
+    for k, t in tensors.items():
+        if k.startswith("h_") and t.is_cuda:
+            raise ValueError("%s must be a host tensor" % k)
+        if (k.startswith("d_") or k == "W_vocab") and not t.is_cuda:
+            raise ValueError("%s must be a device tensor" % k)
+        setattr(st, k, t.data_ptr())
+    st.workspace_bytes = tensors["d_workspace"].numel() * tensors["d_workspace"].element_size()
+    return st
+
+
+def arrol_prune_rebatch_host(ctx: Context, step: _HostStep, stream=None):
+    _check(load_library().arrol_prune_rebatch_host(ctx.handle, C.byref(step), _stream(stream)),
+           "arrol_prune_rebatch_host")

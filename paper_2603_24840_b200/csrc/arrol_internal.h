@@ -12,6 +12,7 @@ struct arrol_ctx {
     uint32_t* h_status;        // pinned host mirror used by arrol_poll_status
     float* d_scratch;          // MLP-head partial sums: [ARROL_SCRATCH_FLOATS]
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
+    unsigned long long launches;   // kernels launched through this context (host-side count)
 };
 
 constexpr int ARROL_MAX_MLP_N = 65536;       // rollouts per arrol_score_partial call with an MLP head

@@ -183,6 +183,7 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     scan_adv_kernel<<<1, SCAN_THREADS, 0, s>>>(keep, lengths, N, G, rewards, (double)eps, ddof,
                                                dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
                                                ctx->d_status);
+    ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     const bool any_token_output = dst_tokens || dst_rows || tok_adv || tok_seq;
     if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
@@ -203,6 +204,7 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
         d_num, cu_seqlens, survivor_idx, src_tok_off, src_tokens, static_cast<const uint4*>(src_rows),
         vec_per_row, adv, dst_capacity_tokens, tile_rows, dst_tokens, static_cast<uint4*>(dst_rows), tok_adv,
         tok_seq);
+    ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
 }

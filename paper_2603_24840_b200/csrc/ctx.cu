@@ -43,6 +43,7 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->h_status = nullptr;
     ctx->d_scratch = nullptr;
     ctx->encode_tiled = nullptr;
+    ctx->launches = 0;
     bool ok = cudaMalloc(&ctx->d_status, 256) == cudaSuccess &&
               cudaMemset(ctx->d_status, 0, 256) == cudaSuccess &&
               cudaMallocHost(&ctx->h_status, 64) == cudaSuccess &&
@@ -72,6 +73,8 @@ extern "C" int arrol_destroy(arrol_ctx* ctx) {
     delete ctx;
     return ARROL_OK;
 }
+
+extern "C" int64_t arrol_launch_count(arrol_ctx* ctx) { return ctx ? (int64_t)ctx->launches : -1; }
 
 extern "C" int arrol_poll_status(arrol_ctx* ctx, void* stream, uint32_t* dev_status_bits) {
     if (!ctx) return ARROL_ERR_INVALID_ARG;

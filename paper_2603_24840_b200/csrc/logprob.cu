@@ -470,12 +470,14 @@ extern "C" int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const voi
     int64_t grid = m_tiles * p.splits;
     if (grid > ctx->sm_count) grid = ctx->sm_count;
     token_logprob_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
+    ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     if (p.splits > 1) {
         int64_t blocks = (T_max + 255) / 256;
         if (blocks > (int64_t)ctx->sm_count * 8) blocks = (int64_t)ctx->sm_count * 8;
         combine_splits_kernel<<<(unsigned)blocks, 256, 0, s>>>(p.partial, targets, d_T, T_max, V, p.splits, logp,
                                                               lse, ctx->d_status);
+        ctx->launches += 1;
         ARROL_CUDA_OK(cudaGetLastError());
     }
     return ARROL_OK;

@@ -217,6 +217,7 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
         score_linear_kernel<T><<<blocks, 32 * warps_per_block, 0, s>>>(
             hid, row_stride, row_index, N, head->d, static_cast<const T*>(head->W1),
             static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q);
+        ctx->launches += 1;
     } else {
         const int h_tiles = (head->h + TH - 1) / TH;
         dim3 grid((N + TM - 1) / TM, h_tiles);
@@ -227,6 +228,7 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
         score_mlp_finish_kernel<T><<<(N + 255) / 256, 256, 0, s>>>(ctx->d_scratch, N, h_tiles,
                                                                   static_cast<const T*>(head->b2), B, q_lut,
                                                                   score, prob, bin, q);
+        ctx->launches += 2;
     }
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;

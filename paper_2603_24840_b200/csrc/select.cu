@@ -77,6 +77,7 @@ extern "C" int arrol_select(arrol_ctx* ctx, const float* q, int32_t P, int32_t G
     if (!guard.ok) return ARROL_ERR_CUDA;
     select_kernel<<<(warps + warps_per_block - 1) / warps_per_block, 32 * warps_per_block, 0,
                     (cudaStream_t)stream>>>(q, P, G, K, rho, seg, keep);
+    ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
 }
