@@ -204,6 +204,34 @@ typedef struct arrol_host_step {
 /* Returns ARROL_OK, a validation/launch error, or the device status translated as by arrol_poll_status. */
 int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* step, void* stream);
 
+/* ---- MLP-head scoring that allocates nothing ---------------------------------------------------------
+ * (The paper has no counterpart to this call: it is a packaging variant of arrol_score_partial, added for
+ * integration, and computes exactly the same outputs for an MLP head.)
+ *
+ * Who needs it: code that may not allocate device memory at the point where it scores rollouts.  Examples are a
+ * serving or training process whose memory plan is frozen after start-up (all device memory already handed to
+ * a pool or arena, so a raw cudaMalloc may fail or is forbidden by policy), a plug-in loaded into a host
+ * application that owns the device heap, and latency-critical loops where an allocation's implicit device
+ * synchronisation is not acceptable.  arrol_create allocates (status word, scratch), so such callers cannot
+ * even make a context; this call therefore takes no context and runs on the calling thread's current device.
+ *
+ * How: the per-tile partial scores that arrol_score_partial keeps in the context scratch live here in a fixed
+ * array inside the library image (128 KiB of device global memory on every GPU that loads the library, held
+ * until the process exits).  Limits that follow from the fixed size: head->h > 0 (MLP head only),
+ * N <= 4096 rollouts and head->h <= 512 per call; larger values return ARROL_ERR_UNSUPPORTED.  All other
+ * arguments, layouts, alignment rules and outputs are those of arrol_score_partial.
+ *
+ * The first call on each device resolves the array's device address (a one-time, per-device set-up inside this
+ * call, guarded by a mutex); make that first call before starting any stream capture on that device.
+ * The call itself never calls cudaMalloc, cudaFree or any allocating library routine.
+ * Every call on a device shares the one array, which keeps whatever the previous call left in it.  Nothing in it
+ * has to start at zero: each call overwrites every entry it later reads.  Two calls that overlap in time on the
+ * same GPU (different streams, or different host threads) race on the array and corrupt each other's scores;
+ * issue them on one stream or order them yourself. */
+int arrol_score_partial_static(const void* hidden, int64_t row_stride_elems, const int64_t* row_index, int32_t N,
+                               const arrol_head* head, const arrol_calib* calib, float* score, float* prob,
+                               int32_t* bin, float* q, void* stream);
+
 /* Number of kernels this context has launched so far (host-side count; -1 for a NULL context). */
 int64_t arrol_launch_count(arrol_ctx* ctx);
 

@@ -21,6 +21,7 @@ EXPORTS = [
     "arrol_version", "arrol_status_string", "arrol_create", "arrol_destroy", "arrol_poll_status",
     "arrol_calib_counts", "arrol_build_q_lut", "arrol_score_partial", "arrol_select", "arrol_compact",
     "arrol_token_logprob_workspace", "arrol_token_logprob", "arrol_prune_rebatch_host", "arrol_launch_count",
+    "arrol_score_partial_static",
 ]
 
 
@@ -93,6 +94,10 @@ def load_library():
                                         C.c_size_t, C.c_void_p]
     lib.arrol_prune_rebatch_host.argtypes = [C.c_void_p, C.POINTER(_HostStep), C.c_void_p]
     lib.arrol_prune_rebatch_host.restype = C.c_int
+    lib.arrol_score_partial_static.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.POINTER(_Head),
+                                               C.POINTER(_Calib), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_void_p]
+    lib.arrol_score_partial_static.restype = C.c_int
     lib.arrol_launch_count.argtypes = [C.c_void_p]
     lib.arrol_launch_count.restype = C.c_int64
     for fn in ("arrol_create", "arrol_destroy", "arrol_poll_status", "arrol_calib_counts", "arrol_build_q_lut",
@@ -279,3 +284,23 @@ def make_host_step(scalars: dict, head: dict, q_lut: Optional[torch.Tensor], ten
 def arrol_prune_rebatch_host(ctx: Context, step: _HostStep, stream=None):
     _check(load_library().arrol_prune_rebatch_host(ctx.handle, C.byref(step), _stream(stream)),
            "arrol_prune_rebatch_host")
+
+
+def arrol_score_partial_static(hidden: torch.Tensor, head: dict, N: int, score: torch.Tensor, prob: torch.Tensor,
+                               q: torch.Tensor, bin: Optional[torch.Tensor] = None,
+                               row_index: Optional[torch.Tensor] = None, q_lut: Optional[torch.Tensor] = None,
+                               row_stride: Optional[int] = None, stream=None):
+    """MLP-head scoring for callers that may not allocate device memory (a frozen memory plan, a host
+    application that owns the device heap, a latency-critical loop): no context, no allocation; the scratch is
+    a fixed 128 KiB array inside the library.  Limits: MLP head only, N <= 4096, h <= 512.  Runs on the current
+    device; calls that overlap on one GPU race on the shared scratch.  The first call per device does a one-time
+    address look-up and should come before any stream capture."""
+    hs = _Head()
+    _fill_head(hs, _dtype_code(hidden), hidden.shape[-1], head)
+    cs = _Calib()
+    cs.B = 0 if q_lut is None else q_lut.shape[0]
+    cs.q_lut = None if q_lut is None else q_lut.data_ptr()
+    stride = hidden.stride(-2) if row_stride is None else int(row_stride)
+    _check(load_library().arrol_score_partial_static(_ptr(hidden), stride, _ptr(row_index), int(N), C.byref(hs),
+                                                     C.byref(cs), _ptr(score), _ptr(prob), _ptr(bin), _ptr(q),
+                                                     _stream(stream)), "arrol_score_partial_static")

@@ -268,3 +268,83 @@ extern "C" int arrol_score_partial(arrol_ctx* ctx, const void* hidden, int64_t r
     return launch_score<__nv_bfloat16>(ctx, hidden, row_stride_elems, row_index, N, head, B, q_lut, score, prob,
                                        bin, q, s);
 }
+
+// ---- MLP-head scoring without any allocation --------------------------------------------------------------
+// Same kernels as above, but the per-tile partial scores live in a fixed array in device global memory that
+// is part of the library image, so this entry point needs neither an arrol_ctx (whose creation allocates)
+// nor any other allocation.  Every device that loads the library carries the array until the process exits.
+#include <mutex>
+
+constexpr int ARROL_STATIC_MAX_N = 4096;                       // rollouts per call
+constexpr int ARROL_STATIC_MAX_H = 512;                        // hidden units of the head
+constexpr int ARROL_STATIC_MAX_TILES = ARROL_STATIC_MAX_H / ARROL_MLP_TH;
+constexpr int ARROL_STATIC_MAX_DEVICES = 64;
+
+// [h_tiles][N] partial scores, 128 KiB.  In host code this name is only a handle for the runtime; the device
+// address is obtained per device with cudaGetSymbolAddress below.
+static __device__ __align__(256) float g_static_mlp_partial[ARROL_STATIC_MAX_TILES * ARROL_STATIC_MAX_N];
+
+static std::mutex g_static_setup_mutex;
+static float* g_static_partial_addr[ARROL_STATIC_MAX_DEVICES] = {nullptr};
+
+extern "C" int arrol_score_partial_static(const void* hidden, int64_t row_stride_elems, const int64_t* row_index,
+                                          int32_t N, const arrol_head* head, const arrol_calib* calib,
+                                          float* score, float* prob, int32_t* bin, float* q, void* stream) {
+    if (!head || N < 0) return ARROL_ERR_INVALID_ARG;
+    if (N == 0) return ARROL_OK;
+    if (!hidden || !score || !prob || !q || !head->W1 || !head->w2) return ARROL_ERR_INVALID_ARG;
+    if (head->dtype != ARROL_F32 && head->dtype != ARROL_BF16) return ARROL_ERR_INVALID_ARG;
+    if (head->d <= 0 || head->h <= 0) return ARROL_ERR_INVALID_ARG;      // MLP head only
+    if (head->d % 8 != 0 || head->h % 4 != 0) return ARROL_ERR_UNSUPPORTED;
+    if (N > ARROL_STATIC_MAX_N || head->h > ARROL_STATIC_MAX_H) return ARROL_ERR_UNSUPPORTED;   // beyond the fixed scratch
+    const int esz = head->dtype == ARROL_F32 ? 4 : 2;
+    if (row_stride_elems < head->d) return ARROL_ERR_INVALID_ARG;
+    if (!arrol_aligned(hidden, 16) || !arrol_aligned(head->W1, 16) || (row_stride_elems * esz) % 16 != 0)
+        return ARROL_ERR_INVALID_ARG;
+    int B = 0;
+    const float* q_lut = nullptr;
+    if (calib) {
+        if (calib->q_lut && calib->B <= 0) return ARROL_ERR_INVALID_ARG;
+        B = calib->B > 0 ? calib->B : 0;
+        q_lut = calib->q_lut;
+    }
+
+    // One-time set-up per device, on the caller's current device: resolve the array's device address.
+    int dev = -1;
+    ARROL_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= ARROL_STATIC_MAX_DEVICES) return ARROL_ERR_UNSUPPORTED;
+    float* partial = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_setup_mutex);
+        if (!g_static_partial_addr[dev]) {
+            float* addr = nullptr;
+            ARROL_CUDA_OK(cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_static_mlp_partial));
+            if (!addr) return ARROL_ERR_CUDA;
+            g_static_partial_addr[dev] = addr;
+        }
+        partial = g_static_partial_addr[dev];
+    }
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h_tiles = (head->h + TH - 1) / TH;
+    dim3 grid((N + TM - 1) / TM, h_tiles);
+    // The tile kernel writes every entry [tile][i], i < N, that the finishing kernel reads, so nothing left in
+    // the array by an earlier call is ever read and nothing needs clearing.
+    if (head->dtype == ARROL_F32) {
+        score_mlp_tile_kernel<float><<<grid, 256, 0, s>>>(
+            static_cast<const float*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
+            static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
+            static_cast<const float*>(head->w2), partial);
+        score_mlp_finish_kernel<float><<<(N + 255) / 256, 256, 0, s>>>(
+            partial, N, h_tiles, static_cast<const float*>(head->b2), B, q_lut, score, prob, bin, q);
+    } else {
+        score_mlp_tile_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(
+            static_cast<const __nv_bfloat16*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
+            static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
+            static_cast<const __nv_bfloat16*>(head->w2), partial);
+        score_mlp_finish_kernel<__nv_bfloat16><<<(N + 255) / 256, 256, 0, s>>>(
+            partial, N, h_tiles, static_cast<const __nv_bfloat16*>(head->b2), B, q_lut, score, prob, bin, q);
+    }
+    ARROL_CUDA_OK(cudaGetLastError());
+    return ARROL_OK;
+}
