@@ -4,10 +4,11 @@
 // Kernel 1 (one block): stable partition by a block-wide prefix sum over (kept flag, kept length):
 //   survivor_idx, cu_seqlens, {S, T}, and per-survivor advantages (fp64 statistics over the kept rollouts of
 //   the group, in index order, rounded once to fp32).
-// Kernel 2 (persistent grid): moves the survivors' rows.  A tile is a run of consecutive destination rows;
-//   one thread per row finds its survivor by binary search in cu_seqlens and writes the per-token outputs
-//   (token id, survivor ordinal, advantage); then the whole block streams the row payload with 16-byte
-//   loads/stores.  T is read from device memory, so there is no host synchronisation between the kernels.
+// Kernel 2 (one wave of persistent blocks): moves the survivors' rows.  Each block owns a contiguous run of
+//   destination tiles (~32 KB of rows each); one thread per row finds its survivor (binary search once per
+//   block, then a forward walk in cu_seqlens) and writes the per-token outputs (token id, survivor ordinal,
+//   advantage); the block then streams the tile's payload with 16-byte loads/stores, eight in flight per thread.
+//   T is read from device memory, so there is no host synchronisation between the kernels.
 #include "arrol_internal.h"
 
 namespace {
@@ -98,59 +99,80 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 }
 
 constexpr int GATHER_THREADS = 256;
-constexpr int MAX_TILE_ROWS = 256;
 
-// tile_rows: destination rows per tile (<= MAX_TILE_ROWS); vec_per_row = row_bytes / 16 (0 without payload)
-__global__ void __launch_bounds__(GATHER_THREADS)
+// Largest s in [lo, hi) with cu_seqlens[s] <= t, given cu_seqlens[lo] <= t < cu_seqlens[hi].  Taking the last
+// such s skips zero-length survivors.
+__device__ __forceinline__ int find_survivor(const int64_t* __restrict__ cu_seqlens, int lo, int hi, int64_t t) {
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(cu_seqlens + mid) <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+constexpr int MAX_TILE_ROWS = 256;
+constexpr int BATCH_VECS = 8 * GATHER_THREADS;   // 16-byte vectors a block moves per pass: 32 KB
+
+// tile_rows: destination rows per tile (<= MAX_TILE_ROWS); vec_per_row = row_bytes / 16 (0 without payload).
+// Every block owns a contiguous run of tiles: it locates its first row's survivor once by binary search and
+// then only walks forward, so the per-tile look-up is a load or two instead of a search.
+__global__ void __launch_bounds__(GATHER_THREADS, 5)
 gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_seqlens,
               const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
               const int32_t* __restrict__ src_tokens, const uint4* __restrict__ src_rows, int vec_per_row,
               const float* __restrict__ adv, int64_t capacity, int tile_rows, int32_t* __restrict__ dst_tokens,
               uint4* __restrict__ dst_rows, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
     __shared__ int64_t src_row_of[MAX_TILE_ROWS];
+    __shared__ int s_first[2];               // survivor of the first row of the current / next tile
     const int S = (int)d_num[0];
     const int64_t T = d_num[1];
-    if (T > capacity || S <= 0) return;      // capacity overflow was recorded by the scan kernel
+    if (T > capacity || S <= 0 || T <= 0) return;      // capacity overflow was recorded by the scan kernel
     const int64_t n_tiles = (T + tile_rows - 1) / tile_rows;
-    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const int64_t tiles_per_block = (n_tiles + gridDim.x - 1) / gridDim.x;
+    const int64_t tile_begin = (int64_t)blockIdx.x * tiles_per_block;
+    const int64_t tile_end = min(n_tiles, tile_begin + tiles_per_block);
+    if (tile_begin >= tile_end) return;
+    if (threadIdx.x == 0) s_first[0] = find_survivor(cu_seqlens, 0, S, tile_begin * tile_rows);
+    __syncthreads();
+    int parity = 0;
+    for (int64_t tile = tile_begin; tile < tile_end; ++tile, parity ^= 1) {
         const int64_t t0 = tile * tile_rows;
         const int rows_here = (int)min((int64_t)tile_rows, T - t0);
+        const int s0 = s_first[parity];
         for (int r = threadIdx.x; r < rows_here; r += GATHER_THREADS) {
             const int64_t t = t0 + r;
-            // largest s with cu_seqlens[s] <= t  (zero-length survivors are skipped by taking the last one)
-            int lo = 0, hi = S;                 // invariant: cu[lo] <= t < cu[hi]
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if (cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+            int s = s0;
+            for (int steps = 0; __ldg(cu_seqlens + s + 1) <= t; ++steps) {
+                if (steps == 8) { s = find_survivor(cu_seqlens, s, S, t); break; }   // many short survivors
+                ++s;
             }
-            const int64_t src = src_tok_off[survivor_idx[lo]] + (t - cu_seqlens[lo]);
+            const int64_t src = __ldg(src_tok_off + __ldg(survivor_idx + s)) + (t - __ldg(cu_seqlens + s));
             src_row_of[r] = src;
-            if (dst_tokens) dst_tokens[t] = src_tokens[src];
-            if (tok_seq) tok_seq[t] = lo;
-            if (tok_adv) tok_adv[t] = adv[lo];
+            if (dst_tokens) dst_tokens[t] = __ldg(src_tokens + src);
+            if (tok_seq) tok_seq[t] = s;
+            if (tok_adv) tok_adv[t] = __ldg(adv + s);
+            if (r == rows_here - 1) s_first[parity ^ 1] = s;
         }
+        __syncthreads();
         if (vec_per_row > 0) {
-            __syncthreads();
-            const int64_t total = (int64_t)rows_here * vec_per_row;
+            const int total = rows_here * vec_per_row;
             uint4* dst = dst_rows + t0 * vec_per_row;
-            int64_t v = threadIdx.x;
-            // eight 16-byte loads in flight per thread
-            for (; v + 7 * GATHER_THREADS < total; v += 8 * GATHER_THREADS) {
+            // eight 16-byte loads in flight per thread; the last pass of a tile is predicated
+            for (int v0 = 0; v0 < total; v0 += BATCH_VECS) {
                 uint4 buf[8];
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const int64_t vv = v + u * GATHER_THREADS;
-                    const int r = (int)(vv / vec_per_row);
-                    const int c = (int)(vv - (int64_t)r * vec_per_row);
-                    buf[u] = ld_stream(src_rows + src_row_of[r] * vec_per_row + c);
+                    const int vv = v0 + u * GATHER_THREADS + threadIdx.x;
+                    if (vv < total) {
+                        const int r = vv / vec_per_row;
+                        buf[u] = ld_stream(src_rows + src_row_of[r] * vec_per_row + (vv - r * vec_per_row));
+                    }
                 }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) st_stream(dst + v + u * GATHER_THREADS, buf[u]);
-            }
-            for (; v < total; v += GATHER_THREADS) {
-                const int r = (int)(v / vec_per_row);
-                const int c = (int)(v - (int64_t)r * vec_per_row);
-                st_stream(dst + v, ld_stream(src_rows + src_row_of[r] * vec_per_row + c));
+                for (int u = 0; u < 8; ++u) {
+                    const int vv = v0 + u * GATHER_THREADS + threadIdx.x;
+                    if (vv < total) st_stream(dst + vv, buf[u]);
+                }
             }
             __syncthreads();
         }
@@ -191,13 +213,19 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     const int vec_per_row = src_rows ? row_bytes / 16 : 0;
     int tile_rows = MAX_TILE_ROWS;
     if (vec_per_row > 0) {
-        // about 32 KB of payload per tile: eight 16-byte vectors per thread per pass
-        tile_rows = (8 * GATHER_THREADS) / vec_per_row;
+        // as many whole rows as fit one 32 KB pass (rows larger than that take several passes each)
+        tile_rows = BATCH_VECS / vec_per_row;
         if (tile_rows < 1) tile_rows = 1;
         if (tile_rows > MAX_TILE_ROWS) tile_rows = MAX_TILE_ROWS;
     }
+    if ((int64_t)tile_rows * vec_per_row > INT32_MAX) return ARROL_ERR_UNSUPPORTED;
     const int64_t max_tiles = (dst_capacity_tokens + tile_rows - 1) / tile_rows;
-    int64_t blocks = (int64_t)ctx->sm_count * 8;
+    // Exactly one wave: every block owns an equal contiguous share of the destination, so a partial second wave
+    // would leave SMs idle at the end.
+    int resident = 0;
+    ARROL_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, gather_kernel, GATHER_THREADS, 0));
+    if (resident < 1) resident = 1;
+    int64_t blocks = (int64_t)ctx->sm_count * resident;
     if (blocks > max_tiles) blocks = max_tiles;
     if (blocks < 1) blocks = 1;
     gather_kernel<<<(unsigned)blocks, GATHER_THREADS, 0, s>>>(

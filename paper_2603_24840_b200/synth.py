@@ -61,6 +61,10 @@ WORKLOADS: Dict[str, Workload] = {
                  "beta_bernoulli", 3, degenerate_frac=0.30),
         Workload("qwen3-8b-dapo", 256, 16, 8, 1024, 8192, ("lognormal", 3000.0, 0.35), 4096, 151936, "bf16", 512,
                  "beta_bernoulli", 4),
+        # Small case for profiler captures: the Llama-shaped d and V on ~75k survivor tokens, so that inputs are
+        # larger than L2 while the device holds about 1.5 GB and a log-prob launch lasts ~25 ms.
+        Workload("profile-small", 48, 8, 4, 256, 512, ("uniform", 256, 512), 2048, 128256, "bf16", 0,
+                 "beta_bernoulli", 9),
         # Mid-size case for CPU-only tests: several tiles and ragged tails, seconds on the host.
         Workload("mini", 6, 8, 4, 16, 96, ("uniform", 16, 96), 192, 1000, "bf16", 24,
                  "beta_bernoulli", 7, degenerate_frac=0.34),

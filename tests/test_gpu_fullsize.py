@@ -1,0 +1,95 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times (PruneRebatch.step()):
+outputs the oracle can compute cheaply are compared in full (scores, selection, scan, advantages, token ids);
+the hidden-row payload and the token log-probs are compared on sampled rows, plus properties that hold at any
+size (every packed row equals its source row; lse >= the target logit; exp(logp) in (0, 1])."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_24840_b200 import binding as B
+from paper_2603_24840_b200 import synth
+from paper_2603_24840_b200.pipeline import PruneRebatch, host_inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _fullsize(name, n_logp_rows):
+    w = synth.WORKLOADS[name]
+    inp = host_inputs(w)                       # big tensors are generated on the device
+    pr = PruneRebatch(w, inputs=inp)
+    pr.step()
+    torch.cuda.synchronize()
+    assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+    oa = lambda t: None if t is None else synth.as_oracle_array(t)
+    head = inp["head"]
+    off = inp["src_tok_off"]
+    ridx = off[:-1] + (w.cutoff - 1)
+
+    # a1/a2: the N rows the head reads, copied back for the oracle
+    x_cut = pr.hidden_score[torch.from_numpy(ridx).to(pr.dev)].cpu()
+    s_ref = oracle.head_score(oa(x_cut), oa(head["W1"]), oa(head["b1"]), oa(head["w2"]), oa(head["b2"]), h=w.h)
+    p_ref, b_ref, _ = oracle.prob_map(s_ref, inp["q_lut"])
+    prob = pr.prob.cpu().numpy()
+    assert np.abs(pr.score.cpu().numpy() - s_ref).max() <= 1e-3
+    assert np.abs(prob - p_ref).max() <= 1e-3
+    bins = pr.bin.cpu().numpy()
+    assert np.array_equal(bins, np.array([oracle.bin_index(float(v), w.B) for v in prob]))
+    q_gpu = pr.q.cpu().numpy()
+    assert np.array_equal(q_gpu, inp["q_lut"][bins])
+
+    # a3: selection, bit-exact, on the oracle's q and on the q the pipeline consumed
+    _, _, q_ref = oracle.prob_map(s_ref, inp["q_lut"])
+    keep_on_oracle_q = torch.empty(w.N, dtype=torch.uint8, device=pr.dev)
+    B.arrol_select(pr.ctx, torch.from_numpy(q_ref.astype(np.float32)).to(pr.dev), w.P, w.G, w.K, w.rho,
+                   keep_on_oracle_q)
+    assert np.array_equal(keep_on_oracle_q.cpu().numpy(), oracle.select(q_ref.astype(np.float32), w.P, w.G, w.K, w.rho))
+    keep_ref = oracle.select(q_gpu, w.P, w.G, w.K, w.rho)
+    assert np.array_equal(pr.keep.cpu().numpy(), keep_ref)
+
+    # a4/a6: scan and advantages in full
+    idx, cu, S, T = oracle.survivor_scan(keep_ref, inp["lengths"])
+    assert pr.counts() == (S, T) and S == w.S and T <= pr.cap
+    assert np.array_equal(pr.survivor_idx.cpu().numpy()[:S], idx)
+    assert np.array_equal(pr.cu_seqlens.cpu().numpy()[:S + 1], cu)
+    adv_ref = oracle.advantages(inp["rewards"], keep_ref, w.G)
+    adv = pr.adv.cpu().numpy()[:S]
+    assert np.abs(adv - adv_ref).max() <= 1e-5
+    rew_kept = inp["rewards"][keep_ref == 1].reshape(w.P, w.K)
+    flat = (rew_kept.min(1) == rew_kept.max(1))
+    assert np.all(adv.reshape(w.P, w.K)[flat] == 0.0)          # all-0 / all-1 survivor sets: exactly zero
+
+    # a5: token ids in full; per-token bookkeeping; hidden rows: every packed row equals its source row
+    dt_ref, _, seq_ref = oracle.gather(idx, cu, off[:-1], inp["src_tokens"])
+    assert np.array_equal(pr.dst_tokens.cpu().numpy()[:T], dt_ref)
+    assert np.array_equal(pr.tok_seq.cpu().numpy()[:T], seq_ref)
+    assert np.array_equal(pr.tok_adv.cpu().numpy()[:T], adv[seq_ref])
+    src_row = torch.from_numpy(off[:-1][idx][seq_ref] + (np.arange(T) - cu[:-1][seq_ref])).to(pr.dev)
+    step = 1 << 16
+    for t0 in range(0, T, step):
+        t1 = min(T, t0 + step)
+        assert torch.equal(pr.dst_rows[t0:t1], pr.src_rows[src_row[t0:t1]])
+
+    # a7: sampled rows against the fp64 oracle; first/last row of every 16th survivor, the forced edge ids, the
+    # last (partial) token tile, the rest uniform at random
+    g = np.random.default_rng(w.seed)
+    rows = np.unique(np.concatenate([[0, T - 1], cu[:-1][::16], cu[1:][::16] - 1, np.arange(T - T % 128, T)[:4],
+                                     np.flatnonzero(dt_ref[:4096] >= (w.V // 256) * 256)[:4],
+                                     g.integers(0, T, size=n_logp_rows)])).astype(np.int64)
+    rows = rows[(rows >= 0) & (rows < T)]
+    H = pr.dst_rows[torch.from_numpy(rows).to(pr.dev)].cpu()
+    lp_ref, lse_ref = oracle.token_logprob(oa(H), oa(pr.W_vocab.cpu()), dt_ref[rows])
+    logp = pr.logp.cpu().numpy()[:T]
+    lse = pr.lse.cpu().numpy()[:T]
+    assert np.abs(logp[rows] - lp_ref).max() <= 2e-3
+    assert np.abs(lse[rows] - lse_ref).max() <= 2e-3
+    assert np.all(np.isfinite(logp)) and np.all(logp <= 1e-6) and np.all(logp > -60.0)
+    pr.ctx.close()
+
+
+def test_llama_3_2_1b_shaped():
+    _fullsize("llama-3.2-1b", 40)
+
+
+def test_qwen3_1_7b_shaped():
+    _fullsize("qwen3-1.7b", 24)
