@@ -27,9 +27,19 @@ sys.path.insert(0, ROOT)
 METRIC = "survivor_logprob_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM traffic of one token_logprob launch per survivor token, from the ncu capture summarised under profiles/
-# (bytes read + written divided by the tokens of the captured launch); None until a capture exists.
-LOGPROB_DRAM_BYTES_PER_TOKEN = None
+# DRAM traffic of one token_logprob launch per survivor token at d = 2048, V = 128256 (two vocabulary splits), from
+# the ncu capture summarised in profiles/token_logprob_kernel_profile-small.md: (4.531 GB read + 7.5 MB written) /
+# 75,382 tokens.  At fixed d, V and split count the traffic grows in proportion to the tokens of the launch.
+LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256): 60200.0}
+
+
+def logprob_traffic(w, T, splits, sm_count):
+    """DRAM bytes of one token_logprob launch: the ncu capture scaled by tokens where one exists for this (d, V),
+    else the model the capture confirmed: every wave of resident blocks streams its W_vocab split once."""
+    per_tok = LOGPROB_DRAM_BYTES_PER_TOKEN.get((w.d, w.V))
+    if per_tok is not None:
+        return per_tok * T, "ncu capture on profile-small scaled by tokens"
+    return 2.0 * w.d * (1.0 + w.V * splits / (sm_count * 128.0)) * T, "model 2d(1 + V*splits/(SMs*128)) per token"
 
 
 def load_peaks():
@@ -268,6 +278,24 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     prune_tokens_only_us = a.elapsed_time(b) / K * 1e3
 
+    # scoring kernel on its own: the linear head streamed over every source row (HBM-bound: d*e bytes per row);
+    # the MLP head on the workload's own N rollouts (fp32-ALU-bound: 2*d*h flops per row)
+    n_score = min(pr.T_src, 1 << 20) if w.h == 0 else w_rank.N
+    so = [torch.empty(n_score, dtype=torch.float32, device=pr.dev) for _ in range(3)]
+    ridx = None if w.h == 0 else pr.row_index
+    for _ in range(3):
+        B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, n_score, so[0], so[1], so[2], row_index=ridx,
+                              q_lut=pr.q_lut)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(K):
+        B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, n_score, so[0], so[1], so[2], row_index=ridx,
+                              q_lut=pr.q_lut)
+    b.record(stream)
+    torch.cuda.synchronize()
+    score_ms = a.elapsed_time(b) / K
+    del so
+
     # ---- e2e: host buffers through arrol_prune_rebatch_host ----
     if args.skip_e2e:
         e2e = {"ms_per_step": float("nan"), "h2d": 0, "d2h": 0}
@@ -297,12 +325,15 @@ def run_ours(args, w):
         achieved = flops / (logp_ms * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
         gather_bytes = 2.0 * T * w.d * 2 + 8.0 * T
+        ws_bytes = pr.workspace.numel()
+        splits = max(1, (ws_bytes - 256) // (16 * pr.cap)) if ws_bytes > 256 else 1
+        traffic, traffic_src = logprob_traffic(w, T, splits, torch.cuda.get_device_properties(local).multi_processor_count)
         roofline = {
             "kernel": "token_logprob_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
             "unit": "TFLOP/s", "frac": achieved / peak,
             "peak_source": "%s bf16 sustained (kernel timed inside a long step)" % peaks["source"],
             "frac_of_burst": achieved / float(peaks["bf16_tflops"]), "frac_of_nominal_2250": achieved / 2250.0,
-            "traffic": None if LOGPROB_DRAM_BYTES_PER_TOKEN is None else LOGPROB_DRAM_BYTES_PER_TOKEN * T,
+            "traffic": traffic, "traffic_source": traffic_src, "vocab_splits": int(splits),
             "algorithmic_flops_per_launch": flops,
             "launch_ms": logp_ms,
         }
@@ -334,6 +365,22 @@ def run_ours(args, w):
                                  "unit": "GB/s", "frac": compact_gbs / float(peaks["hbm_gbs"]),
                                  "algorithmic_bytes_per_launch": gather_bytes},
         }
+        esz = pr.hidden_score.element_size()
+        props = torch.cuda.get_device_properties(local)
+        if w.h == 0:
+            gbs = n_score * w.d * esz / (score_ms * 1e-3) / 1e9
+            out["score_roofline"] = {"kernel": "score_linear_kernel", "bound": "hbm", "rows": int(n_score),
+                                     "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+                                     "frac": gbs / float(peaks["hbm_gbs"]), "launch_ms": score_ms,
+                                     "note": "linear head streamed over consecutive source rows; the step itself "
+                                             "scores only N = %d rows (launch-latency bound)" % w_rank.N}
+        else:
+            tfs = 2.0 * n_score * w.d * w.h / (score_ms * 1e-3) / 1e12
+            alu_peak = 2.0 * 128 * props.multi_processor_count * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+            out["score_roofline"] = {"kernel": "score_mlp_tile_kernel", "bound": "alu", "rows": int(n_score),
+                                     "achieved": tfs, "peak": alu_peak, "unit": "TFLOP/s", "frac": tfs / alu_peak,
+                                     "launch_ms": score_ms,
+                                     "note": "fp32 FMA roof = 2 x 128 lanes x SMs x max SM clock"}
         if not args.no_cpu_baseline and world == 1:
             v, sample, cores, _ = oracle_step_rate(w, args.cpu_budget)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}

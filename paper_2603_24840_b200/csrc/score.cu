@@ -1,9 +1,11 @@
 // arrol_score_partial: quality head on the hidden state at the detection length, sigmoid, bin index and
 // posterior lookup (Section 4.2; Appendix A.4).
 //
-// Linear head: HBM-bound row reduction, one warp per rollout, 16-byte loads, shuffle reduction, with the
+// Linear head: HBM-bound row reduction, one warp per rollout, 16-byte loads (eight in flight per lane), shuffle
+// reduction, with the
 // probability map fused into lane 0's epilogue.
-// MLP head: fp32 SIMT register-tiled contraction (64 rollouts x 64 hidden units per block) with the bias,
+// MLP head: fp32 SIMT register-tiled contraction (64 rollouts x 64 hidden units per block, 8 x 4 per thread,
+// next K chunk prefetched into registers) with the bias,
 // exact GELU and the w2 dot product fused into the tile epilogue; per-tile partial scores go to the context
 // scratch and a finishing kernel adds them in a fixed order and applies the probability map.
 #include <cuda_bf16.h>
@@ -19,6 +21,11 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162flo
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {
     static constexpr int N = 4;
+    using Raw = float4;
+    __device__ static __forceinline__ Raw load_raw(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+    __device__ static __forceinline__ float dot(const Raw& a, const Raw& b, float acc) {
+        acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc); acc = fmaf(a.z, b.z, acc); return fmaf(a.w, b.w, acc);
+    }
     __device__ static __forceinline__ void load(const float* p, float (&out)[4]) {
         float4 v = __ldg(reinterpret_cast<const float4*>(p));
         out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
@@ -26,6 +33,17 @@ template <> struct Vec16<float> {
 };
 template <> struct Vec16<__nv_bfloat16> {
     static constexpr int N = 8;
+    using Raw = uint4;
+    __device__ static __forceinline__ Raw load_raw(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+    __device__ static __forceinline__ float dot(const Raw& a, const Raw& b, float acc) {
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {   // a bf16 is the upper half of a binary32
+            acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
+            acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
+        }
+        return acc;
+    }
     __device__ static __forceinline__ void load(const __nv_bfloat16* p, float (&out)[8]) {
         uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -65,26 +83,20 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
     const T* x = hidden + row * row_stride;
     const int nvec = d / VN;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    int c = lane;
-    // four independent 16-byte loads in flight per lane
-    for (; c + 96 < nvec; c += 128) {
-        float xv[4][VN], wv[4][VN];
+    // eight independent 16-byte loads of x (and of w) in flight per lane: a 4 KB row is one round trip
+    for (int c0 = lane; c0 < nvec; c0 += 256) {
+        typename Vec16<T>::Raw xr[8], wr[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            Vec16<T>::load(x + (int64_t)(c + 32 * u) * VN, xv[u]);
-            Vec16<T>::load(w + (int64_t)(c + 32 * u) * VN, wv[u]);
+        for (int u = 0; u < 8; ++u) {
+            const int c = c0 + 32 * u;
+            if (c < nvec) {
+                xr[u] = Vec16<T>::load_raw(x + (int64_t)c * VN);
+                wr[u] = Vec16<T>::load_raw(w + (int64_t)c * VN);
+            }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-#pragma unroll
-            for (int e = 0; e < VN; ++e) acc[u] = fmaf(xv[u][e], wv[u][e], acc[u]);
-    }
-    for (; c < nvec; c += 32) {
-        float xv[VN], wv[VN];
-        Vec16<T>::load(x + (int64_t)c * VN, xv);
-        Vec16<T>::load(w + (int64_t)c * VN, wv);
-#pragma unroll
-        for (int e = 0; e < VN; ++e) acc[0] = fmaf(xv[e], wv[e], acc[0]);
+        for (int u = 0; u < 8; ++u)
+            if (c0 + 32 * u < nvec) acc[u & 3] = Vec16<T>::dot(xr[u], wr[u], acc[u & 3]);
     }
     float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
 #pragma unroll
@@ -96,76 +108,102 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
 }
 
 // ---- MLP head ---------------------------------------------------------------------------------------
-// Block tile: TM = 64 rollouts x TH = 64 hidden units, K chunks of 32; 256 threads, 4 x 4 outputs each.
-constexpr int TM = 64, TH = ARROL_MLP_TH, TK = 32, PAD = 4;
+// Block tile: TM = 64 rollouts x TH = 64 hidden units, K chunks of 32; 128 threads, 8 x 4 outputs each.
+// The next K chunk is fetched from global memory into registers while the current one is multiplied out of
+// shared memory (two shared buffers, one barrier per chunk).
+constexpr int TM = 64, TH = ARROL_MLP_TH, TK = 32, PAD = 4, MLP_THREADS = 128;
 
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(MLP_THREADS)
 score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index,
                       int N, int d, int h, const T* __restrict__ W1, const T* __restrict__ b1,
                       const T* __restrict__ w2, float* __restrict__ partial /* [h_tiles][N] */) {
     constexpr int VN = Vec16<T>::N;
-    constexpr int VPR = TK / VN;               // 16-byte vectors per tile row per K chunk
-    __shared__ __align__(16) float xs[TK][TM + PAD];
-    __shared__ __align__(16) float ws[TK][TH + PAD];
+    constexpr int VPR = TK / VN;                       // 16-byte vectors per tile row per K chunk
+    constexpr int NV = TM * VPR / MLP_THREADS;         // vectors per thread per operand per chunk (2 or 4)
+    static_assert(TM == TH && (TM * VPR) % MLP_THREADS == 0, "tile / thread mapping");
+    __shared__ __align__(16) float xs[2][TK][TM + PAD];
+    __shared__ __align__(16) float ws[2][TK][TH + PAD];
 
     const int m0 = blockIdx.x * TM, j0 = blockIdx.y * TH;
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;   // tx: hidden units, ty: rollouts
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;   // tx: 4 hidden units each, ty: 8 rollouts each
 
-    float acc[4][4];
+    // Global -> register staging.  Vector v of a chunk covers tile row (v % TM), K offset (v / TM) * VN, so that
+    // the lanes of a warp write consecutive shared-memory columns (no bank conflicts).
+    const T* xrow[NV];
+    const T* wrow[NV];
+    int kofs[NV], rr[NV];
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int i = 0; i < NV; ++i) {
+        const int v = threadIdx.x + i * MLP_THREADS;
+        rr[i] = v % TM;
+        kofs[i] = (v / TM) * VN;
+        const int m = m0 + rr[i], j = j0 + rr[i];
+        xrow[i] = nullptr;
+        wrow[i] = nullptr;
+        if (m < N) xrow[i] = hidden + (row_index ? row_index[m] : (int64_t)m) * row_stride;
+        if (j < h) wrow[i] = W1 + (int64_t)j * d;
+    }
+    float xreg[NV][VN], wreg[NV][VN];
+    auto fetch = [&](int k0) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int k = k0 + kofs[i];
+            if (xrow[i] && k < d) Vec16<T>::load(xrow[i] + k, xreg[i]);
+            else {
+#pragma unroll
+                for (int e = 0; e < VN; ++e) xreg[i][e] = 0.f;
+            }
+            if (wrow[i] && k < d) Vec16<T>::load(wrow[i] + k, wreg[i]);
+            else {
+#pragma unroll
+                for (int e = 0; e < VN; ++e) wreg[i][e] = 0.f;
+            }
+        }
+    };
+    auto stash = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < NV; ++i)
+#pragma unroll
+            for (int e = 0; e < VN; ++e) {
+                xs[buf][kofs[i] + e][rr[i]] = xreg[i][e];
+                ws[buf][kofs[i] + e][rr[i]] = wreg[i][e];
+            }
+    };
+
+    float acc[8][4];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
-    for (int k0 = 0; k0 < d; k0 += TK) {
-        // stage X[m0..m0+63][k0..k0+31] and W1[j0..j0+63][k0..k0+31] as fp32, k-major
-        for (int v = threadIdx.x; v < TM * VPR; v += 256) {
-            const int r = v / VPR, cv = v % VPR;
-            const int k = k0 + cv * VN;
-            float vals[VN];
-            const int m = m0 + r;
-            if (m < N && k < d) {
-                const int64_t row = row_index ? row_index[m] : (int64_t)m;
-                Vec16<T>::load(hidden + row * row_stride + k, vals);
-            } else {
-#pragma unroll
-                for (int e = 0; e < VN; ++e) vals[e] = 0.f;
-            }
-#pragma unroll
-            for (int e = 0; e < VN; ++e) xs[cv * VN + e][r] = vals[e];
-        }
-        for (int v = threadIdx.x; v < TH * VPR; v += 256) {
-            const int r = v / VPR, cv = v % VPR;
-            const int k = k0 + cv * VN;
-            float vals[VN];
-            const int j = j0 + r;
-            if (j < h && k < d) {
-                Vec16<T>::load(W1 + (int64_t)j * d + k, vals);
-            } else {
-#pragma unroll
-                for (int e = 0; e < VN; ++e) vals[e] = 0.f;
-            }
-#pragma unroll
-            for (int e = 0; e < VN; ++e) ws[cv * VN + e][r] = vals[e];
-        }
-        __syncthreads();
+    fetch(0);
+    stash(0);
+    __syncthreads();
+    int buf = 0;
+    for (int k0 = 0; k0 < d; k0 += TK, buf ^= 1) {
+        const bool more = k0 + TK < d;
+        if (more) fetch(k0 + TK);
 #pragma unroll
         for (int k = 0; k < TK; ++k) {
-            const float4 xa = *reinterpret_cast<const float4*>(&xs[k][ty * 4]);
-            const float4 wb = *reinterpret_cast<const float4*>(&ws[k][tx * 4]);
-            const float xr[4] = {xa.x, xa.y, xa.z, xa.w};
+            const float4 xa = *reinterpret_cast<const float4*>(&xs[buf][k][ty * 8]);
+            const float4 xb = *reinterpret_cast<const float4*>(&xs[buf][k][ty * 8 + 4]);
+            const float4 wb = *reinterpret_cast<const float4*>(&ws[buf][k][tx * 4]);
+            const float xr[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
             const float wr[4] = {wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
-            for (int a = 0; a < 4; ++a)
+            for (int a = 0; a < 8; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(xr[a], wr[b], acc[a][b]);
         }
+        if (more) stash(buf ^ 1);      // the other buffer was last read before the previous barrier
         __syncthreads();
     }
 
     // epilogue: u + b1 -> exact GELU -> dot with w2 over this tile's hidden units
-    float part[4] = {0.f, 0.f, 0.f, 0.f};
+    float part[8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a) part[a] = 0.f;
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
         const int j = j0 + tx * 4 + b;
@@ -173,22 +211,22 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
             const float bj = b1 ? to_f32(b1[j]) : 0.f;
             const float wj = to_f32(w2[j]);
 #pragma unroll
-            for (int a = 0; a < 4; ++a) {
+            for (int a = 0; a < 8; ++a) {
                 const float u = acc[a][b] + bj;
                 const float g = 0.5f * u * (1.0f + erff(u * 0.70710678118654752440f));
                 part[a] = fmaf(wj, g, part[a]);
             }
         }
     }
-    // the 16 threads of one rollout quadruple are lanes (ty & 1) * 16 + tx of a warp: reduce over tx
+    // the 16 threads that share a group of 8 rollouts are one half-warp: reduce over tx
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+    for (int a = 0; a < 8; ++a)
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) part[a] += __shfl_xor_sync(0xffffffffu, part[a], o, 16);
     if (tx == 0) {
 #pragma unroll
-        for (int a = 0; a < 4; ++a) {
-            const int m = m0 + ty * 4 + a;
+        for (int a = 0; a < 8; ++a) {
+            const int m = m0 + ty * 8 + a;
             if (m < N) partial[(int64_t)blockIdx.y * N + m] = part[a];
         }
     }
@@ -221,7 +259,7 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
     } else {
         const int h_tiles = (head->h + TH - 1) / TH;
         dim3 grid((N + TM - 1) / TM, h_tiles);
-        score_mlp_tile_kernel<T><<<grid, 256, 0, s>>>(hid, row_stride, row_index, N, head->d, head->h,
+        score_mlp_tile_kernel<T><<<grid, MLP_THREADS, 0, s>>>(hid, row_stride, row_index, N, head->d, head->h,
                                                      static_cast<const T*>(head->W1),
                                                      static_cast<const T*>(head->b1),
                                                      static_cast<const T*>(head->w2), ctx->d_scratch);
@@ -331,14 +369,14 @@ extern "C" int arrol_score_partial_static(const void* hidden, int64_t row_stride
     // The tile kernel writes every entry [tile][i], i < N, that the finishing kernel reads, so nothing left in
     // the array by an earlier call is ever read and nothing needs clearing.
     if (head->dtype == ARROL_F32) {
-        score_mlp_tile_kernel<float><<<grid, 256, 0, s>>>(
+        score_mlp_tile_kernel<float><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const float*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
             static_cast<const float*>(head->w2), partial);
         score_mlp_finish_kernel<float><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const float*>(head->b2), B, q_lut, score, prob, bin, q);
     } else {
-        score_mlp_tile_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(
+        score_mlp_tile_kernel<__nv_bfloat16><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const __nv_bfloat16*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
             static_cast<const __nv_bfloat16*>(head->w2), partial);
