@@ -206,9 +206,8 @@ def run_ours(args, w):
     import torch
     import torch.distributed as dist
     from paper_2603_24840_b200 import binding as B
-    from paper_2603_24840_b200 import synth
-    from paper_2603_24840_b200.pipeline import PruneRebatch, host_inputs
-    import dataclasses
+    from paper_2603_24840_b200 import dist_util, synth
+    from paper_2603_24840_b200.pipeline import PruneRebatch
 
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
@@ -220,7 +219,7 @@ def run_ours(args, w):
     C = args.prompt_chunks if args.prompt_chunks > 0 else auto_prompt_chunks(w)
     while w.P % C != 0:
         C += 1
-    w_rank = dataclasses.replace(w, P=w.P // C, seed=w.seed + 1000 * rank)
+    w_rank = dist_util.shard_workload(w, rank, world, prompt_chunks=C)
 
     pr = PruneRebatch(w_rank, device=local, with_rows=True)
     stream = torch.cuda.current_stream()
@@ -307,14 +306,8 @@ def run_ours(args, w):
             e2e = {"ms_per_step": float("nan"), "h2d": 0, "d2h": 0}
 
     # ---- reduce over ranks ----
-    t_total = torch.tensor([total_ms, e2e["ms_per_step"]], dtype=torch.float64, device="cuda")
-    tok = torch.tensor([float(T) * C], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t_total, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
-    total_ms_max = float(t_total[0])
-    e2e_ms_max = float(t_total[1]) * C   # the host-buffer leg runs one chunk per call
-    tokens_all = float(tok[0])
+    total_ms_max, e2e_ms_max, tokens_all = dist_util.reduce_timings(total_ms, e2e["ms_per_step"], float(T) * C, "cuda")
+    e2e_ms_max *= C                      # the host-buffer leg runs one chunk per call
 
     if rank == 0:
         peaks = load_peaks()

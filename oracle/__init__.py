@@ -212,3 +212,61 @@ def token_logprob(hidden, W, targets, rows=None, inv_temp: float = 1.0):
     if rc != 0:
         raise MemoryError("oracle_token_logprob could not allocate its scratch")
     return logp, lse
+
+
+class ScoreBuffers:
+    """Positive / negative sliding buffers of normalised scores (Appendix A.4), FIFO of `cap` entries each."""
+
+    def __init__(self, cap: int):
+        self.cap = int(cap)
+        self.pos = np.zeros(cap, dtype=np.float64)
+        self.neg = np.zeros(cap, dtype=np.float64)
+        self.state = np.zeros(4, dtype=np.int64)      # head_pos, n_pos, head_neg, n_neg
+
+    def push(self, sprime, y):
+        sprime = np.ascontiguousarray(sprime, dtype=np.float64)
+        y = np.ascontiguousarray(y, dtype=np.uint8)
+        st = self.state
+        P64 = C.POINTER(C.c_int64)
+        base = st.ctypes.data
+        ptr = lambda i: C.cast(base + 8 * i, P64)
+        lib().oracle_buffer_push(_p(self.pos), ptr(0), ptr(1), _p(self.neg), ptr(2), ptr(3), C.c_int64(self.cap),
+                                 _p(sprime), _p(y), C.c_int64(sprime.shape[0]))
+
+    def contents(self):
+        """(positive scores oldest..newest, negative scores oldest..newest)"""
+        hp, n_p, hn, n_n = (int(v) for v in self.state)
+        pos = np.array([self.pos[(hp + i) % self.cap] for i in range(n_p)])
+        neg = np.array([self.neg[(hn + i) % self.cap] for i in range(n_n)])
+        return pos, neg
+
+    def counts(self, B: int):
+        pos, neg = self.contents()
+        s = np.concatenate([pos, neg])
+        y = np.concatenate([np.ones(len(pos), np.uint8), np.zeros(len(neg), np.uint8)])
+        return calib_counts(s, y, B)
+
+
+def solve_delta(cpos, cneg, q_lut, kappa=0.5, lam=0.5, rho=0.5, p_min=0.05, p_max=0.95, iters=64) -> float:
+    cpos = np.ascontiguousarray(cpos, dtype=np.int64)
+    cneg = np.ascontiguousarray(cneg, dtype=np.int64)
+    q_lut = np.ascontiguousarray(q_lut, dtype=np.float32)
+    f = lib().oracle_solve_delta
+    f.restype = C.c_double
+    return float(f(_p(cpos), _p(cneg), _p(q_lut), C.c_int(q_lut.shape[0]), C.c_double(kappa), C.c_double(lam),
+                   C.c_double(rho), C.c_double(p_min), C.c_double(p_max), C.c_int(iters)))
+
+
+def select_stochastic(q, u, delta, eligible=None, kappa=0.5, lam=0.5, rho=0.5, p_min=0.05, p_max=0.95):
+    """Returns (keep uint8 [N], p float64 [N])."""
+    q = np.ascontiguousarray(q, dtype=np.float32)
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    N = q.shape[0]
+    if eligible is not None:
+        eligible = np.ascontiguousarray(eligible, dtype=np.uint8)
+    keep = np.empty(N, dtype=np.uint8)
+    p = np.empty(N, dtype=np.float64)
+    lib().oracle_select_stochastic(_p(q), _p(u), _p(eligible), C.c_int64(N), C.c_double(kappa), C.c_double(delta),
+                                   C.c_double(lam), C.c_double(rho), C.c_double(p_min), C.c_double(p_max),
+                                   _p(keep), _p(p))
+    return keep, p

@@ -285,3 +285,79 @@ int oracle_token_logprob(const void* hidden, const void* W, int dtype, const int
     }
     return err;
 }
+
+/* ---------------------------------------------------------------------------------------------
+ * Deployed stochastic pruning rule (Appendix A.4, Eq. "survival"; Algorithm 1, backend).
+ *
+ * Sliding buffers: positives and negatives are kept in two first-in-first-out buffers of `cap` normalised
+ * scores each; pushing into a full buffer drops its oldest entry.  The histogram counts c_b^+ / c_b^- are the
+ * counts over what the buffers hold (Eq. "count").
+ * buf_pos / buf_neg: [cap] ring storage of s', head_* = index of the oldest entry, n_* = entries held.
+ * --------------------------------------------------------------------------------------------- */
+void oracle_buffer_push(double* buf_pos, int64_t* head_pos, int64_t* n_pos, double* buf_neg, int64_t* head_neg,
+                        int64_t* n_neg, int64_t cap, const double* sprime, const uint8_t* y, int64_t n) {
+    for (int64_t k = 0; k < n; ++k) {
+        double* buf = y[k] ? buf_pos : buf_neg;
+        int64_t* head = y[k] ? head_pos : head_neg;
+        int64_t* cnt = y[k] ? n_pos : n_neg;
+        if (*cnt < cap) {
+            buf[(*head + *cnt) % cap] = sprime[k];
+            *cnt += 1;
+        } else {
+            buf[*head] = sprime[k];          /* overwrite the oldest, which becomes the newest */
+            *head = (*head + 1) % cap;
+        }
+    }
+}
+
+/* Survival probability p = clip(kappa + delta + lambda (rho - q), p_min, p_max). */
+static double survival_of(double q, double kappa, double delta, double lambda, double rho, double p_min,
+                          double p_max) {
+    double p = kappa + delta;
+    p = p + lambda * (rho - q);
+    if (p < p_min) p = p_min;
+    if (p > p_max) p = p_max;
+    return p;
+}
+
+/* delta by bisection so that the expected keep rate under the buffer distribution equals kappa:
+ *   E[p] = sum_b w_b clip(kappa + delta + lambda (rho - q_b), p_min, p_max) = kappa,
+ *   w_b = (c_b^+ + c_b^-) / n   (every buffered rollout counts once; q_b is the posterior of its bin).
+ * E[p] is non-decreasing in delta.  Bracket [-(1 + lambda), 1 + lambda], `iters` halvings (64 in the library);
+ * the midpoint moves up when E[p] < kappa.  Empty buffers give delta = 0.  Sums run over bins in index order. */
+double oracle_solve_delta(const int64_t* cpos, const int64_t* cneg, const float* q_lut, int B, double kappa,
+                          double lambda, double rho, double p_min, double p_max, int iters) {
+    double n = 0.0;
+    for (int b = 0; b < B; ++b) n = n + (double)(cpos[b] + cneg[b]);
+    if (!(n > 0.0)) return 0.0;
+    double lo = -(1.0 + lambda), hi = 1.0 + lambda;
+    for (int it = 0; it < iters; ++it) {
+        double mid = 0.5 * (lo + hi);
+        double e = 0.0;
+        for (int b = 0; b < B; ++b) {
+            double wb = (double)(cpos[b] + cneg[b]);
+            e = e + wb * survival_of((double)q_lut[b], kappa, mid, lambda, rho, p_min, p_max);
+        }
+        e = e / n;
+        if (e < kappa) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+/* Per-rollout decision: a rollout that has reached the detection length (eligible) survives iff u < p_i;
+ * a rollout that ended earlier is never evaluated and is kept.  p (optional) receives p_i (1 for the
+ * ineligible). u in [0,1) are the uniforms drawn for this step, passed in. */
+void oracle_select_stochastic(const float* q, const float* u, const uint8_t* eligible, int64_t N, double kappa,
+                              double delta, double lambda, double rho, double p_min, double p_max,
+                              uint8_t* keep, double* p) {
+    for (int64_t i = 0; i < N; ++i) {
+        if (eligible && !eligible[i]) {
+            keep[i] = 1;
+            if (p) p[i] = 1.0;
+            continue;
+        }
+        double pi = survival_of((double)q[i], kappa, delta, lambda, rho, p_min, p_max);
+        if (p) p[i] = pi;
+        keep[i] = ((double)u[i] < pi) ? 1 : 0;
+    }
+}
