@@ -149,6 +149,45 @@ int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab,
                         int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                         float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- Online calibrator and the deployed stochastic rule (Appendix A.4; Algorithm 1, backend) ----------
+ * The calibrator state lives in ONE caller-provided device buffer of arrol_calib_state_bytes(B, cap) bytes
+ * (16-byte aligned): two first-in-first-out rings of `cap` bin indices (positive / negative rollouts), their
+ * histogram counts c_b^+ / c_b^-, the posterior table q_lut [B] and the bias delta.  B <= 1024.
+ *
+ * arrol_calib_init: empty rings, zero counts, q_lut = 0.5, delta = 0.
+ * arrol_calib_update: pushes the rollouts i < N with mask[i] != 0 (all when mask is NULL) in index order: rollout i
+ *   goes to the positive ring if rewards[i] > 0.5, else to the negative ring, as bin index bin[i] (the output of
+ *   arrol_score_partial); a full ring drops its oldest entry.  Then rebuilds
+ *     q_b = pi P(b|1) / (pi P(b|1) + (1-pi) P(b|0)),  P(b|Y) = (c_b + alpha) / (sum c + alpha B),  pi = n+/(n+ + n-)
+ *   and solves delta by 64 bisection steps on [-(1+lambda), 1+lambda] so that
+ *     sum_b (c_b^+ + c_b^-) clip(kappa + delta + lambda (rho - q_b), p_min, p_max) / (n+ + n-) = kappa
+ *   (delta = 0 while both rings are empty).  fp64, one rounding per operation, fixed order: reproducible bit for bit.
+ * arrol_calib_q_lut / arrol_calib_delta: device addresses of the table and of delta inside the state (pointer
+ *   arithmetic on the host; no device access), to be passed to arrol_score_partial / arrol_select_stochastic.
+ * arrol_calib_layout: byte offsets {c+, c-, q_lut, ring+, ring-, total} inside the state, for inspection.
+ * arrol_select_stochastic: p_i = clip(kappa + delta + lambda (rho - q_i), p_min, p_max) in fp64;
+ *   keep[i] = (u[i] < p_i), u [N] float uniforms in [0,1) supplied by the caller; rollouts with eligible[i] == 0
+ *   (ended before the detection length, never evaluated) are kept with p = 1.  delta is read from d_delta
+ *   (device) when it is not NULL, else the host value `delta` is used.  p_out [N] float or NULL. */
+typedef struct arrol_survival {
+    double kappa;   /* target keep rate            */
+    double lambda;  /* strength of the correction  */
+    double rho;     /* target positive ratio       */
+    double p_min, p_max;
+} arrol_survival;
+
+size_t arrol_calib_state_bytes(int32_t B, int64_t cap);
+int arrol_calib_layout(int32_t B, int64_t cap, size_t* offsets6 /* host [6] */);
+int arrol_calib_init(arrol_ctx* ctx, void* state, size_t state_bytes, int32_t B, int64_t cap, double alpha,
+                     void* stream);
+int arrol_calib_update(arrol_ctx* ctx, void* state, int32_t B, int64_t cap, const int32_t* bin, const float* rewards,
+                       const uint8_t* mask, int32_t N, const arrol_survival* params, void* stream);
+const float* arrol_calib_q_lut(void* state, int32_t B, int64_t cap);
+const double* arrol_calib_delta(void* state);
+int arrol_select_stochastic(arrol_ctx* ctx, const float* q, const float* u, const uint8_t* eligible, int64_t N,
+                            const arrol_survival* params, const double* d_delta, double delta, uint8_t* keep,
+                            float* p_out, void* stream);
+
 /* ---- Whole step from host buffers (Algorithm 1, frontend lines "filter ... rebatch ... log-probs on R'") --
  * Convenience call for callers whose per-step data lives in host memory: copies the step's inputs to the device
  * staging buffers, runs arrol_score_partial -> arrol_select -> arrol_compact -> arrol_token_logprob on `stream`,

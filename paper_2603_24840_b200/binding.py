@@ -22,6 +22,8 @@ EXPORTS = [
     "arrol_calib_counts", "arrol_build_q_lut", "arrol_score_partial", "arrol_select", "arrol_compact",
     "arrol_token_logprob_workspace", "arrol_token_logprob", "arrol_prune_rebatch_host", "arrol_launch_count",
     "arrol_score_partial_static",
+    "arrol_calib_state_bytes", "arrol_calib_layout", "arrol_calib_init", "arrol_calib_update", "arrol_calib_q_lut",
+    "arrol_calib_delta", "arrol_select_stochastic",
 ]
 
 
