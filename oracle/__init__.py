@@ -23,10 +23,11 @@ F32, BF16, F64 = 0, 1, 2
 
 def build(force: bool = False) -> str:
     """Compile the oracle (plain C, -O2, no fast-math, no FMA contraction, OpenMP over independent units)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    srcs = sorted(os.path.join(_HERE, f) for f in os.listdir(_HERE) if f.endswith(".c"))
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(os.path.getmtime(s) for s in srcs):
         tmp = _LIB + ".%d.tmp" % os.getpid()
-        subprocess.check_call(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
-                               _SRC, "-o", tmp, "-lm"])
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC"] +
+                              srcs + ["-o", tmp, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
