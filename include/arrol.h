@@ -188,6 +188,32 @@ int arrol_select_stochastic(arrol_ctx* ctx, const float* q, const float* u, cons
                             const arrol_survival* params, const double* d_delta, double delta, uint8_t* keep,
                             float* p_out, void* stream);
 
+/* ---- Policy update on the survivors (Section 3: clipped objective; Algorithm 1 "main RL loss", "Backprop") ----
+ * arrol_policy_loss: for every packed survivor token t < T (T, S read from d_num = {S, T}, device):
+ *     r = exp(logp[t] - logp_old[t]),  term = min(r A, clip(r, 1 - eps_low, 1 + eps_high) A),  A = tok_adv[t];
+ *     loss = - sum_t w_t term_t  (+ beta sum_t w_t (exp(ref - logp) - (ref - logp) - 1) when logp_ref != NULL);
+ *     agg_mode 0 (GRPO): w_t = 1 / (S * length of the token's rollout), rollout = tok_seq[t], lengths from cu_seqlens;
+ *     agg_mode 1 (DAPO): w_t = 1 / T.
+ *   Outputs: grad_logp [T_max] float = d loss / d logp (d term / d logp = r A when r A <= clip(r) A, else 0);
+ *   loss: device double [1].  fp32 per token, fp64 fixed-order reduction.  Uses the context scratch: calls on one
+ *   context must be issued on one stream at a time.
+ * arrol_lm_head_backward: given grad_logp [T_max] and lse [T_max] (from arrol_token_logprob on the same inputs),
+ *     dz_{t,v} = grad_logp[t] inv_temperature ([v = targets[t]] - exp(z_{t,v} - lse[t])),  z recomputed on the tensor
+ *     cores;  dH [T_max, d] float = dz W_vocab (rows t >= T are zero or left untouched);  dW [V, d] float = dz^T hidden
+ *     (overwritten).  Positions with targets[t] < 0 or >= V carry no gradient.  dz is rounded to bf16 before the two
+ *     contractions.  hidden, W_vocab, targets, T_max, d_T, d, V as in arrol_token_logprob; dH, dW 16-byte aligned.
+ *   workspace: arrol_lm_head_backward_workspace(ctx, T_max, d, V) bytes, 256-byte aligned (W^T, one chunk of 9,472
+ *   tokens of dz in both orientations, the chunk of hidden transposed): about 4 * 9472 * V + 2 * d * (V + 9472) bytes. */
+int arrol_policy_loss(arrol_ctx* ctx, const float* logp, const float* logp_old, const float* logp_ref,
+                      const float* tok_adv, const int32_t* tok_seq, const int64_t* cu_seqlens, const int64_t* d_num,
+                      int64_t T_max, float eps_low, float eps_high, float beta, int32_t agg_mode, float* grad_logp,
+                      double* loss, void* stream);
+size_t arrol_lm_head_backward_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
+int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                           const float* grad_logp, const float* lse, int64_t T_max, const int64_t* d_T, int32_t d,
+                           int32_t V, float inv_temperature, float* dH, float* dW, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 /* ---- Whole step from host buffers (Algorithm 1, frontend lines "filter ... rebatch ... log-probs on R'") --
  * Convenience call for callers whose per-step data lives in host memory: copies the step's inputs to the device
  * staging buffers, runs arrol_score_partial -> arrol_select -> arrol_compact -> arrol_token_logprob on `stream`,

@@ -1,0 +1,520 @@
+// arrol_lm_head_backward: gradient of the selected-token log-probs through the lm_head (Section 3: the policy
+// update differentiates log pi_theta(o_t | o_<t); Algorithm 1 "Backprop ... on policy").
+//
+//   z = inv_temp H W^T,  logp_t = z_{t,y_t} - lse_t,  given g_t = dL/dlogp_t and lse_t from the forward call:
+//   dz_{t,v} = g_t inv_temp ([v = y_t] - exp(z_{t,v} - lse_t)),   dH = dz W,   dW = dz^T H.
+//
+// The tokens are processed in chunks of TC rows.  Per chunk, three tensor-core kernels with the same
+// TMA -> shared memory -> tcgen05.mma -> tensor memory pipeline as the forward kernel:
+//   dz_kernel      recomputes the chunk's logits tile by tile and turns each accumulator tile into dz (bf16),
+//                  written both as dZ [TC, V] and transposed as dZt [V, TC]
+//   gemm_nt_kernel dH[chunk] = dZ . Wt^T        (M = TC, N = d, K = V;  Wt = W^T, transposed once per call)
+//   gemm_nt_kernel dW       += dZt . Ht^T       (M = V,  N = d, K = TC; Ht = chunk of H transposed)
+// so every contraction is of the K-major x K-major form the forward kernel uses.  The T x V matrix exists only one
+// chunk at a time, in the workspace.
+#include "arrol_internal.h"
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 256;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int TMEM_COLS = 512;
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 4;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int TC = 74 * BM;      // tokens per chunk: 74 token tiles, so that TC/128 x d/256 tiles fill 148 SMs evenly
+
+struct PipeSmem {
+    uint8_t* stage_a;
+    uint8_t* stage_b;
+    uint64_t *full, *empty, *acc_full, *acc_empty, *drain;
+    uint32_t* tmem_slot;
+    volatile uint32_t* abort_flag;
+};
+
+__device__ __forceinline__ PipeSmem carve_smem(uint8_t* smem_raw) {
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    PipeSmem ps;
+    ps.stage_a = smem;
+    ps.stage_b = smem + (size_t)STAGES * A_STAGE_BYTES;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
+    ps.full = bars;
+    ps.empty = bars + STAGES;
+    ps.acc_full = bars + 2 * STAGES;
+    ps.acc_empty = ps.acc_full + 2;
+    ps.drain = ps.acc_empty + 2;
+    ps.tmem_slot = reinterpret_cast<uint32_t*>(ps.drain + 1);
+    ps.abort_flag = ps.tmem_slot + 1;
+    return ps;
+}
+
+// Common prologue: barriers, tensor-memory allocation.  Returns the tensor-memory base address.
+__device__ __forceinline__ uint32_t pipe_setup(const PipeSmem& ps, const CUtensorMap* ma, const CUtensorMap* mb) {
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&ps.full[s], 1); mbar_init(&ps.empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&ps.acc_full[b], 1); mbar_init(&ps.acc_empty[b], EPI_WARPS); }
+        mbar_init(ps.drain, 1);
+        *ps.abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(ma) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(mb) : "memory");
+    }
+    if (warp == 1) {
+        tcgen05_alloc(ps.tmem_slot, TMEM_COLS);
+        tcgen05_relinquish();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    return *ps.tmem_slot;
+}
+
+__device__ __forceinline__ void pipe_teardown(const PipeSmem& ps, uint32_t tmem_base, uint32_t* d_status) {
+    tcgen05_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *ps.abort_flag) atomicOr(d_status, ARROL_DEV_WAIT_EXPIRED);
+    if ((threadIdx.x >> 5) == 1) {
+        tcgen05_fence_after();
+        tcgen05_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// Producer role (one thread): for every work item, for every K step, one A tile (row coordinate ay) and one
+// B tile (row coordinate by).  `coords(item, ay, by)` returns false when the item list is exhausted.
+template <typename Coords>
+__device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensorMap* ma, const CUtensorMap* mb,
+                                              int k_steps, Coords coords) {
+    uint32_t stage = 0, phase = 0, issued = 0;
+    bool ok = true;
+    int ay, by;
+    for (int64_t it = 0; ok && coords(it, ay, by); ++it) {
+        for (int ks = 0; ks < k_steps; ++ks) {
+            if (!mbar_wait(&ps.empty[stage], phase ^ 1u, ps.abort_flag)) { ok = false; break; }
+            mbar_expect_tx(&ps.full[stage], STAGE_BYTES);
+            tma_load_2d(ps.stage_a + (size_t)stage * A_STAGE_BYTES, ma, ks * BK, ay, &ps.full[stage]);
+            tma_load_2d(ps.stage_b + (size_t)stage * B_STAGE_BYTES, mb, ks * BK, by, &ps.full[stage]);
+            ++issued;
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+    }
+    if (!ok) {   // gave up: let the copies already issued land before shared memory goes away (bounded)
+        const uint32_t pending = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
+        uint32_t s = stage, ph = phase;
+        for (uint32_t i = 0; i < pending; ++i) {
+            if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+            for (uint32_t spin = 0; spin < SPIN_LIMIT; ++spin)
+                if (mbar_try_wait(&ps.full[s], ph)) break;
+        }
+    }
+}
+
+// MMA role (one thread): n_items accumulator tiles of k_steps K steps each, alternating the two accumulators.
+__device__ __forceinline__ void mma_loop(const PipeSmem& ps, uint32_t tmem_base, int64_t n_items, int k_steps) {
+    constexpr uint32_t idesc = make_idesc(BM, BN);
+    uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (int64_t it = 0; it < n_items && ok; ++it) {
+        if (!mbar_wait(&ps.acc_empty[acc], acc_phase ^ 1u, ps.abort_flag)) { ok = false; break; }
+        tcgen05_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int ks = 0; ks < k_steps; ++ks) {
+            if (!mbar_wait(&ps.full[stage], phase, ps.abort_flag)) { ok = false; break; }
+            tcgen05_fence_after();
+            const uint64_t a_desc = make_smem_desc(smem_u32(ps.stage_a + (size_t)stage * A_STAGE_BYTES));
+            const uint64_t b_desc = make_smem_desc(smem_u32(ps.stage_b + (size_t)stage * B_STAGE_BYTES));
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+                tcgen05_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                 (ks | k) != 0 ? 1u : 0u);
+            tcgen05_commit(&ps.empty[stage]);
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tcgen05_commit(&ps.acc_full[acc]);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+    if (!ok) {
+        tcgen05_commit(ps.drain);
+        for (uint32_t spin = 0; spin < SPIN_LIMIT; ++spin)
+            if (mbar_try_wait(ps.drain, 0u)) break;
+    }
+}
+
+__device__ __forceinline__ int64_t live_tokens(const int64_t* d_T, int64_t T_max) {
+    int64_t T = T_max;
+    if (d_T) { const int64_t t = *d_T; T = t < 0 ? 0 : (t < T ? t : T); }
+    return T;
+}
+
+// ---- dz: recompute logits, write the softmax gradient of one token chunk --------------------------------------
+struct DzParams {
+    const int32_t* targets;
+    const float* grad_logp;
+    const float* lse;
+    const int64_t* d_T;
+    int64_t T_max, t0;        // chunk = tokens [t0, t0 + TC)
+    int d, V;
+    int64_t ldz;              // row pitch of dZ (V rounded up to 8)
+    int splits, chunks_per_split;
+    float scale2, inv_temp;
+    __nv_bfloat16* dZ;        // [TC, ldz]
+    __nv_bfloat16* dZt;       // [V, TC]
+    uint32_t* d_status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const DzParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const PipeSmem ps = carve_smem(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t T = live_tokens(p.d_T, p.T_max);
+    if (p.t0 >= T) return;                                  // chunk past the live tokens (uniform for the grid)
+    const int64_t items = (int64_t)(TC / BM) * p.splits;
+    const int k_steps = (p.d + BK - 1) / BK;
+    const int total_chunks = (p.V + BN - 1) / BN;
+    const uint32_t tmem_base = pipe_setup(ps, &map_h, &map_w);
+
+    // work item -> (token tile, vocabulary range); the accumulator tiles of one item are its vocabulary chunks
+    auto item_range = [&](int64_t item, int& m_tile, int& c0, int& c1) {
+        m_tile = (int)(item / p.splits);
+        const int split = (int)(item % p.splits);
+        c0 = split * p.chunks_per_split;
+        c1 = min(c0 + p.chunks_per_split, total_chunks);
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int64_t item = blockIdx.x;
+            int m_tile = 0, c = 0, c1 = 0;
+            bool have = false;
+            producer_loop(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
+                while (!have || c >= c1) {
+                    if (have) item += gridDim.x;
+                    if (item >= items) return false;
+                    item_range(item, m_tile, c, c1);
+                    have = true;
+                }
+                ay = (int)(p.t0 + (int64_t)m_tile * BM);
+                by = c * BN;
+                ++c;
+                return true;
+            });
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            int64_t n_tiles = 0;
+            for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+                int m_tile, c0, c1;
+                item_range(item, m_tile, c0, c1);
+                n_tiles += max(c1 - c0, 0);
+            }
+            mma_loop(ps, tmem_base, n_tiles, k_steps);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            int m_tile, c0, c1;
+            item_range(item, m_tile, c0, c1);
+            const int row_in_chunk = m_tile * BM + row_in_tile;
+            const int64_t t = p.t0 + row_in_chunk;
+            int y = -1;
+            float coef = 0.f, lse2 = 0.f;
+            if (t < T) {
+                y = p.targets[t];
+                if (y >= 0 && y < p.V) {
+                    coef = p.grad_logp[t] * p.inv_temp;
+                    lse2 = p.lse[t] * 1.44269504088896340736f;
+                } else {
+                    y = -1;
+                }
+            }
+            __nv_bfloat16* zrow = p.dZ + (int64_t)row_in_chunk * p.ldz;
+            for (int c = c0; c < c1 && ok; ++c) {
+                ok = mbar_wait(&ps.acc_full[acc], acc_phase, ps.abort_flag);
+                ok = __all_sync(0xffffffffu, ok) != 0;
+                if (!ok) break;
+                tcgen05_fence_after();
+#pragma unroll 1
+                for (int piece = 0; piece < BN / 32; ++piece) {
+                    const int pc0 = c * BN + piece * 32;
+                    if (pc0 >= p.V) break;
+                    float v[32];
+                    tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        // dz = coef ([v = y] - 2^(z log2e - lse log2e)); coef = 0 for rows that carry no gradient
+                        float d0 = -coef * ex2_approx(fmaf(v[j], p.scale2, -lse2));
+                        float d1 = -coef * ex2_approx(fmaf(v[j + 1], p.scale2, -lse2));
+                        if (pc0 + j == y) d0 += coef;
+                        if (pc0 + j + 1 == y) d1 += coef;
+                        if (coef == 0.f) { d0 = 0.f; d1 = 0.f; }      // also guards 0 * inf from stale lse values
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(d0, d1);
+                        packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
+                    }
+                    const int n_valid = min(32, p.V - pc0);
+                    if (n_valid == 32 && (p.ldz & 7) == 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(zrow + pc0);
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4)
+                            dst[q4] = make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < n_valid) {
+                                const uint32_t w = packed[j >> 1];
+                                reinterpret_cast<uint16_t*>(zrow)[pc0 + j] = (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu));
+                            }
+                        }
+                    }
+                    // transposed copy: for a fixed vocabulary row the 32 lanes write 32 consecutive tokens (64 bytes)
+                    uint16_t* zt = reinterpret_cast<uint16_t*>(p.dZt) + (int64_t)pc0 * TC + row_in_chunk;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (j < n_valid) {
+                            const uint32_t w = packed[j >> 1];
+                            zt[(int64_t)j * TC] = (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu));
+                        }
+                    }
+                }
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ps.acc_empty[acc]);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    }
+    pipe_teardown(ps, tmem_base, p.d_status);
+}
+
+// ---- generic C[M,N] (+)= A[M,K] B[N,K]^T, bf16 operands K-major, fp32 result -------------------------------------
+struct GemmParams {
+    int M, N, K;
+    float* C;
+    int64_t ldc;
+    int accumulate;           // 1: C += A B^T, 0: C = A B^T
+    const int64_t* d_T;       // the launch is skipped when t0 >= live tokens
+    int64_t T_max, t0;
+    uint32_t* d_status;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_nt_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const PipeSmem ps = carve_smem(smem_raw);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (p.t0 >= live_tokens(p.d_T, p.T_max)) return;
+    const int m_tiles = (p.M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
+    const int64_t items = (int64_t)m_tiles * n_tiles;
+    const int k_steps = (p.K + BK - 1) / BK;
+    const uint32_t tmem_base = pipe_setup(ps, &map_a, &map_b);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            producer_loop(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
+                const int64_t item = blockIdx.x + it * gridDim.x;
+                if (item >= items) return false;
+                ay = (int)(item / n_tiles) * BM;       // consecutive blocks share the A panel, walk the B panels
+                by = (int)(item % n_tiles) * BN;
+                return true;
+            });
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const int64_t mine = items > blockIdx.x ? (items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+            mma_loop(ps, tmem_base, mine, k_steps);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            const int row = (int)(item / n_tiles) * BM + quarter * 32 + lane;
+            const int col0 = (int)(item % n_tiles) * BN;
+            ok = mbar_wait(&ps.acc_full[acc], acc_phase, ps.abort_flag);
+            ok = __all_sync(0xffffffffu, ok) != 0;
+            if (!ok) break;
+            tcgen05_fence_after();
+            float* crow = p.C + (int64_t)row * p.ldc;
+#pragma unroll 1
+            for (int piece = 0; piece < BN / 32; ++piece) {
+                const int pc0 = col0 + piece * 32;
+                if (pc0 >= p.N) break;
+                float v[32];
+                tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
+                if (row < p.M) {
+                    if (pc0 + 32 <= p.N && (p.ldc & 3) == 0) {
+                        float4* dst = reinterpret_cast<float4*>(crow + pc0);
+#pragma unroll
+                        for (int q4 = 0; q4 < 8; ++q4) {
+                            float4 o = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+                            if (p.accumulate) {
+                                const float4 c = dst[q4];
+                                o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
+                            }
+                            dst[q4] = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (pc0 + j < p.N) crow[pc0 + j] = p.accumulate ? crow[pc0 + j] + v[j] : v[j];
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ps.acc_empty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+    pipe_teardown(ps, tmem_base, p.d_status);
+}
+
+// ---- bf16 transpose: dst[c, r] = src[r, c] for r < rows_live, zero for rows_live <= r < rows -------------------
+__global__ void transpose_bf16_kernel(const uint16_t* __restrict__ src, int64_t ld_src, int64_t rows, int64_t cols,
+                                      uint16_t* __restrict__ dst, int64_t ld_dst, const int64_t* d_T, int64_t T_max,
+                                      int64_t t0, int use_live) {
+    __shared__ uint16_t tile[64][66];
+    int64_t rows_live = rows;
+    if (use_live) {
+        const int64_t T = live_tokens(d_T, T_max);
+        if (t0 >= T) return;
+        rows_live = min(rows, T - t0);
+    }
+    const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+        const int64_t r = r0 + i, c = c0 + threadIdx.x * 2;
+        uint16_t a = 0, b = 0;
+        if (r < rows_live) {
+            if (c < cols) a = src[r * ld_src + c];
+            if (c + 1 < cols) b = src[r * ld_src + c + 1];
+        }
+        tile[i][threadIdx.x * 2] = a;
+        tile[i][threadIdx.x * 2 + 1] = b;
+    }
+    __syncthreads();
+    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
+        const int64_t c = c0 + i, r = r0 + threadIdx.x * 2;
+        if (c < cols) {
+            if (r < rows) dst[c * ld_dst + r] = tile[threadIdx.x * 2][i];
+            if (r + 1 < rows) dst[c * ld_dst + r + 1] = tile[threadIdx.x * 2 + 1][i];
+        }
+    }
+}
+
+struct BackwardLayout {
+    int64_t ldz;       // V rounded up to 8
+    size_t wt, dz, dzt, ht, total;
+};
+
+BackwardLayout backward_layout(int d, int V) {
+    BackwardLayout L;
+    L.ldz = ((int64_t)V + 7) & ~(int64_t)7;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    size_t o = 0;
+    L.wt = o; o = up(o + (size_t)d * L.ldz * 2);
+    L.dz = o; o = up(o + (size_t)TC * L.ldz * 2);
+    L.dzt = o; o = up(o + (size_t)V * TC * 2);
+    L.ht = o; o = up(o + (size_t)d * TC * 2);
+    L.total = o;
+    return L;
+}
+
+}  // namespace
+
+extern "C" size_t arrol_lm_head_backward_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
+    if (!ctx || T_max <= 0 || d <= 0 || V <= 0) return 0;
+    return backward_layout(d, V).total;
+}
+
+extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                                      const float* grad_logp, const float* lse, int64_t T_max, const int64_t* d_T,
+                                      int32_t d, int32_t V, float inv_temperature, float* dH, float* dW,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
+    if (!ctx || T_max < 0 || d <= 0 || V <= 0 || !(inv_temperature > 0.f)) return ARROL_ERR_INVALID_ARG;
+    if (!dW) return ARROL_ERR_INVALID_ARG;
+    if (d % 8 != 0) return ARROL_ERR_UNSUPPORTED;
+    if (T_max > (int64_t)INT32_MAX - TC) return ARROL_ERR_UNSUPPORTED;
+    ArrolDeviceGuard guard(ctx->device);
+    if (!guard.ok) return ARROL_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    ARROL_CUDA_OK(cudaMemsetAsync(dW, 0, sizeof(float) * (size_t)V * d, s));
+    if (T_max == 0) return ARROL_OK;
+    if (!hidden || !W_vocab || !targets || !grad_logp || !lse || !dH) return ARROL_ERR_INVALID_ARG;
+    if (!arrol_aligned(hidden, 16) || !arrol_aligned(W_vocab, 16) || !arrol_aligned(dH, 16) || !arrol_aligned(dW, 16))
+        return ARROL_ERR_INVALID_ARG;
+    const BackwardLayout L = backward_layout(d, V);
+    if (!workspace || workspace_bytes < L.total || !arrol_aligned(workspace, 256)) return ARROL_ERR_WORKSPACE;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint16_t* Wt = reinterpret_cast<uint16_t*>(ws + L.wt);
+    __nv_bfloat16* dZ = reinterpret_cast<__nv_bfloat16*>(ws + L.dz);
+    __nv_bfloat16* dZt = reinterpret_cast<__nv_bfloat16*>(ws + L.dzt);
+    uint16_t* Ht = reinterpret_cast<uint16_t*>(ws + L.ht);
+
+    ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_nt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+
+    // W^T once per call: [V, d] -> [d, ldz]
+    {
+        dim3 grid((unsigned)((d + 63) / 64), (unsigned)((V + 63) / 64)), block(32, 8);
+        transpose_bf16_kernel<<<grid, block, 0, s>>>(static_cast<const uint16_t*>(W_vocab), d, V, d, Wt, L.ldz, nullptr,
+                                                     0, 0, 0);
+        ctx->launches += 1;
+    }
+    CUtensorMap map_h, map_w, map_dz, map_wt, map_dzt, map_ht;
+    if (make_map(ctx, &map_h, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_dz, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_wt, Wt, (uint64_t)d, (uint64_t)V, (uint64_t)L.ldz, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_dzt, dZt, (uint64_t)V, TC, TC, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_ht, Ht, (uint64_t)d, TC, TC, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+
+    const int total_chunks = (V + BN - 1) / BN;
+    int splits = 1;
+    while ((TC / BM) * splits < ctx->sm_count && splits * 2 <= total_chunks) splits *= 2;
+    const int chunks_per_split = (total_chunks + splits - 1) / splits;
+    splits = (total_chunks + chunks_per_split - 1) / chunks_per_split;
+
+    for (int64_t t0 = 0; t0 < T_max; t0 += TC) {
+        DzParams zp;
+        zp.targets = targets; zp.grad_logp = grad_logp; zp.lse = lse; zp.d_T = d_T; zp.T_max = T_max; zp.t0 = t0;
+        zp.d = d; zp.V = V; zp.ldz = L.ldz; zp.splits = splits; zp.chunks_per_split = chunks_per_split;
+        zp.scale2 = inv_temperature * 1.44269504088896340736f; zp.inv_temp = inv_temperature;
+        zp.dZ = dZ; zp.dZt = dZt; zp.d_status = ctx->d_status;
+        int64_t grid = (int64_t)(TC / BM) * splits;
+        if (grid > ctx->sm_count) grid = ctx->sm_count;
+        dz_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, zp);
+
+        const int64_t rows = (T_max - t0) < TC ? (T_max - t0) : (int64_t)TC;
+        {   // chunk of H transposed, columns past the live tokens zeroed: [rows, d] -> [d, TC]
+            dim3 tg((unsigned)((d + 63) / 64), (unsigned)(TC / 64)), block(32, 8);
+            transpose_bf16_kernel<<<tg, block, 0, s>>>(static_cast<const uint16_t*>(hidden) + t0 * d, d, TC, d, Ht, TC,
+                                                       d_T, T_max, t0, 1);
+        }
+        GemmParams gh;
+        gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0;
+        gh.d_T = d_T; gh.T_max = T_max; gh.t0 = t0; gh.d_status = ctx->d_status;
+        int64_t gh_items = (int64_t)((rows + BM - 1) / BM) * ((d + BN - 1) / BN);
+        gemm_nt_kernel<<<(unsigned)(gh_items < ctx->sm_count ? gh_items : ctx->sm_count), NUM_THREADS, SMEM_BYTES, s>>>(
+            map_dz, map_wt, gh);
+        GemmParams gw;
+        gw.M = V; gw.N = d; gw.K = TC; gw.C = dW; gw.ldc = d; gw.accumulate = 1;
+        gw.d_T = d_T; gw.T_max = T_max; gw.t0 = t0; gw.d_status = ctx->d_status;
+        int64_t gw_items = (int64_t)((V + BM - 1) / BM) * ((d + BN - 1) / BN);
+        gemm_nt_kernel<<<(unsigned)(gw_items < ctx->sm_count ? gw_items : ctx->sm_count), NUM_THREADS, SMEM_BYTES, s>>>(
+            map_dzt, map_ht, gw);
+        ctx->launches += 4;
+        ARROL_CUDA_OK(cudaGetLastError());
+    }
+    return ARROL_OK;
+}
