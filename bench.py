@@ -295,6 +295,14 @@ def run_ours(args, w):
     score_ms = a.elapsed_time(b) / K
     del so
 
+    # ---- policy update on the same survivors (reported separately; not part of `value`) ----
+    update = None
+    if not args.skip_update:
+        try:
+            update = run_update(pr, w_rank, B, torch, K)
+        except (RuntimeError, MemoryError) as exc:
+            print("update leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
+
     # ---- e2e: host buffers through arrol_prune_rebatch_host ----
     if args.skip_e2e:
         e2e = {"ms_per_step": float("nan"), "h2d": 0, "d2h": 0}
@@ -374,6 +382,14 @@ def run_ours(args, w):
                                      "achieved": tfs, "peak": alu_peak, "unit": "TFLOP/s", "frac": tfs / alu_peak,
                                      "launch_ms": score_ms,
                                      "note": "fp32 FMA roof = 2 x 128 lanes x SMs x max SM clock"}
+        if update is not None:
+            upd_flops = 6.0 * T * w.d * w.V
+            out["update"] = {"what": "arrol_policy_loss + arrol_lm_head_backward on the step's survivors "
+                                     "(recompute + dH + dW = 6 T d V flop)",
+                             "ms": update["ms"], "loss_ms": update["loss_ms"], "tokens_per_s": T / (update["ms"] * 1e-3),
+                             "achieved": upd_flops / (update["ms"] * 1e-3) / 1e12, "unit": "TFLOP/s",
+                             "frac": upd_flops / (update["ms"] * 1e-3) / 1e12 / peak, "bound": "tensor",
+                             "workspace_gb": update["ws_gb"]}
         if not args.no_cpu_baseline and world == 1:
             v, sample, cores, _ = oracle_step_rate(w, args.cpu_budget)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
@@ -382,6 +398,44 @@ def run_ours(args, w):
         print(json.dumps(out), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_update(pr, w, B, torch, K):
+    """Times the policy-update calls on the survivors the step produced: loss + gradient, then the lm_head backward."""
+    from paper_2603_24840_b200 import update as U
+    dev, cap = pr.dev, pr.cap
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed + 77)
+    logp_old = pr.logp + 0.05 * torch.randn(cap, generator=gen, device=dev)
+    grad = torch.empty(cap, dtype=torch.float32, device=dev)
+    loss = torch.zeros(1, dtype=torch.float64, device=dev)
+    dH = torch.empty((cap, w.d), dtype=torch.float32, device=dev)
+    dW = torch.empty((w.V, w.d), dtype=torch.float32, device=dev)
+    ws_bytes = U.arrol_lm_head_backward_workspace(pr.ctx, cap, w.d, w.V)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def once():
+        U.arrol_policy_loss(pr.ctx, pr.logp, logp_old, pr.tok_adv, pr.tok_seq, pr.cu_seqlens, pr.d_num, cap, grad, loss,
+                            eps_low=0.2, eps_high=0.28)
+        mid.record(stream)
+        U.arrol_lm_head_backward(pr.ctx, pr.dst_rows, pr.W_vocab, pr.dst_tokens, grad, pr.lse, cap, w.d, w.V, dH, dW, ws,
+                                 d_T=pr.d_num[1:])
+
+    a, mid, b = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    once()
+    torch.cuda.synchronize()
+    n = max(1, min(K, 3))
+    tot = loss_ms = 0.0
+    for _ in range(n):
+        a.record(stream)
+        once()
+        b.record(stream)
+        torch.cuda.synchronize()
+        tot += a.elapsed_time(b)
+        loss_ms += a.elapsed_time(mid)
+    B.arrol_poll_status(pr.ctx)
+    return {"ms": tot / n, "loss_ms": loss_ms / n, "ws_gb": ws_bytes / 1e9}
 
 
 def auto_prompt_chunks(w):
@@ -454,6 +508,7 @@ def main():
     ap.add_argument("--workload", default="llama-3.2-1b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prompt-chunks", type=int, default=0, help="0 = choose from the memory footprint")
+    ap.add_argument("--skip-update", action="store_true", help="leave out the policy-update leg")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
     args = ap.parse_args()
