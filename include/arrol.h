@@ -214,6 +214,16 @@ int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_voc
                            int32_t V, float inv_temperature, float* dH, float* dW, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* ---- Test-time rank-weighted vote (Section 4.4) -----------------------------------------------------------
+ * score [P*G] float: quality-head scores of G completed candidates per prompt (group-major); answer [P*G] int32:
+ * an id of each candidate's final answer (equal ids = equal answers; < 0 = no answer, does not vote).
+ * weight[i] = rank of candidate i inside its group / (G - 1): ranks by ascending score, equal scores in index
+ * order, so the lowest score gets 0 and the highest 1 (a single candidate gets 1).  Every distinct answer sums the
+ * weights of its candidates; winner[p] = the answer with the largest sum (of equal sums the one appearing first),
+ * -1 when the group has no answer; winner_weight[p] = its sum.  Sums are compared as integer rank sums.  G <= 32. */
+int arrol_rank_vote(arrol_ctx* ctx, const float* score, const int32_t* answer, int32_t P, int32_t G, float* weight,
+                    int32_t* winner, float* winner_weight, void* stream);
+
 /* ---- Whole step from host buffers (Algorithm 1, frontend lines "filter ... rebatch ... log-probs on R'") --
  * Convenience call for callers whose per-step data lives in host memory: copies the step's inputs to the device
  * staging buffers, runs arrol_score_partial -> arrol_select -> arrol_compact -> arrol_token_logprob on `stream`,

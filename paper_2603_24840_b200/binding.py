@@ -24,7 +24,7 @@ EXPORTS = [
     "arrol_score_partial_static",
     "arrol_calib_state_bytes", "arrol_calib_layout", "arrol_calib_init", "arrol_calib_update", "arrol_calib_q_lut",
     "arrol_calib_delta", "arrol_select_stochastic",
-    "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward",
+    "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
 ]
 
 
