@@ -214,6 +214,24 @@ int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_voc
                            int32_t V, float inv_temperature, float* dH, float* dW, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* ---- Quality-head training step (Section 4.2; Section 4.3 (iii)) ------------------------------------------
+ * Cross-entropy of the head's logit against the rollout's final reward, gradients into the head only:
+ *     y_i = rewards[i] > 0.5;  over the n rollouts with mask[i] != 0 (all when mask is NULL; e.g. the survivors, the
+ *     only rollouts that ran to a final reward):
+ *     loss = (1/n) sum_i [log(1 + exp(s_i)) - y_i s_i],   ds_i = (sigmoid(s_i) - y_i) / n,
+ *     linear head: dW1 [d] = sum_i ds_i x_i, db1 [1] = sum_i ds_i;
+ *     MLP head:    dw2 [h] = sum_i ds_i gelu(u_i), db2 [1] = sum_i ds_i, du_i = ds_i w2 gelu'(u_i),
+ *                  dW1 [h, d] = du^T X, db1 [h] = sum_i du_i.
+ * hidden / row_stride_elems / row_index / N / head as in arrol_score_partial (the scores are recomputed here).
+ * Outputs are float (loss: device double [1]) and are overwritten; dw2, db2 are ignored for a linear head.
+ * fp32 arithmetic, fixed-order reductions.  N <= 65536.  N == 0 or an all-zero mask gives zero loss and gradients.
+ * workspace: arrol_head_grad_workspace(ctx, N, d, h) bytes, 256-byte aligned.  Uses the context scratch for the
+ * linear head's scores: one stream at a time per context. */
+size_t arrol_head_grad_workspace(arrol_ctx* ctx, int32_t N, int32_t d, int32_t h);
+int arrol_head_grad(arrol_ctx* ctx, const void* hidden, int64_t row_stride_elems, const int64_t* row_index, int32_t N,
+                    const arrol_head* head, const float* rewards, const uint8_t* mask, float* dW1, float* db1,
+                    float* dw2, float* db2, double* loss, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- Test-time rank-weighted vote (Section 4.4) -----------------------------------------------------------
  * score [P*G] float: quality-head scores of G completed candidates per prompt (group-major); answer [P*G] int32:
  * an id of each candidate's final answer (equal ids = equal answers; < 0 = no answer, does not vote).

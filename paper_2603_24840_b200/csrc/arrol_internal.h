@@ -45,3 +45,7 @@ struct ArrolDeviceGuard {
     }
     int cur = -1;
 };
+
+// score.cu: MLP tile pass with optional pre-activation output; partial is [ceil(h / ARROL_MLP_TH)][N].
+int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index, int N,
+                             const arrol_head* head, float* partial, float* u_out, cudaStream_t s);

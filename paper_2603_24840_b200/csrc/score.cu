@@ -117,7 +117,8 @@ template <typename T>
 __global__ void __launch_bounds__(MLP_THREADS)
 score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index,
                       int N, int d, int h, const T* __restrict__ W1, const T* __restrict__ b1,
-                      const T* __restrict__ w2, float* __restrict__ partial /* [h_tiles][N] */) {
+                      const T* __restrict__ w2, float* __restrict__ partial /* [h_tiles][N] */,
+                      float* __restrict__ u_out /* [N][h] pre-activations, or NULL */) {
     constexpr int VN = Vec16<T>::N;
     constexpr int VPR = TK / VN;                       // 16-byte vectors per tile row per K chunk
     constexpr int NV = TM * VPR / MLP_THREADS;         // vectors per thread per operand per chunk (2 or 4)
@@ -213,6 +214,7 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
 #pragma unroll
             for (int a = 0; a < 8; ++a) {
                 const float u = acc[a][b] + bj;
+                if (u_out && m0 + ty * 8 + a < N) u_out[(int64_t)(m0 + ty * 8 + a) * h + j] = u;
                 const float g = 0.5f * u * (1.0f + erff(u * 0.70710678118654752440f));
                 part[a] = fmaf(wj, g, part[a]);
             }
@@ -262,7 +264,7 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
         score_mlp_tile_kernel<T><<<grid, MLP_THREADS, 0, s>>>(hid, row_stride, row_index, N, head->d, head->h,
                                                      static_cast<const T*>(head->W1),
                                                      static_cast<const T*>(head->b1),
-                                                     static_cast<const T*>(head->w2), ctx->d_scratch);
+                                                     static_cast<const T*>(head->w2), ctx->d_scratch, nullptr);
         score_mlp_finish_kernel<T><<<(N + 255) / 256, 256, 0, s>>>(ctx->d_scratch, N, h_tiles,
                                                                   static_cast<const T*>(head->b2), B, q_lut,
                                                                   score, prob, bin, q);
@@ -273,6 +275,26 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
 }
 
 }  // namespace
+
+// Internal: MLP tile pass that also stores the pre-activations u [N][h] (used by the head training step).
+int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index, int N,
+                             const arrol_head* head, float* partial, float* u_out, cudaStream_t s) {
+    const int h_tiles = (head->h + TH - 1) / TH;
+    dim3 grid((N + TM - 1) / TM, h_tiles);
+    if (head->dtype == ARROL_F32)
+        score_mlp_tile_kernel<float><<<grid, MLP_THREADS, 0, s>>>(
+            static_cast<const float*>(hidden), row_stride, row_index, N, head->d, head->h,
+            static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
+            static_cast<const float*>(head->w2), partial, u_out);
+    else
+        score_mlp_tile_kernel<__nv_bfloat16><<<grid, MLP_THREADS, 0, s>>>(
+            static_cast<const __nv_bfloat16*>(hidden), row_stride, row_index, N, head->d, head->h,
+            static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
+            static_cast<const __nv_bfloat16*>(head->w2), partial, u_out);
+    ctx->launches += 1;
+    ARROL_CUDA_OK(cudaGetLastError());
+    return ARROL_OK;
+}
 
 extern "C" int arrol_score_partial(arrol_ctx* ctx, const void* hidden, int64_t row_stride_elems,
                                    const int64_t* row_index, int32_t N, const arrol_head* head,
@@ -372,14 +394,14 @@ extern "C" int arrol_score_partial_static(const void* hidden, int64_t row_stride
         score_mlp_tile_kernel<float><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const float*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
-            static_cast<const float*>(head->w2), partial);
+            static_cast<const float*>(head->w2), partial, nullptr);
         score_mlp_finish_kernel<float><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const float*>(head->b2), B, q_lut, score, prob, bin, q);
     } else {
         score_mlp_tile_kernel<__nv_bfloat16><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const __nv_bfloat16*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
-            static_cast<const __nv_bfloat16*>(head->w2), partial);
+            static_cast<const __nv_bfloat16*>(head->w2), partial, nullptr);
         score_mlp_finish_kernel<__nv_bfloat16><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const __nv_bfloat16*>(head->b2), B, q_lut, score, prob, bin, q);
     }
