@@ -480,9 +480,13 @@ def run_e2e(args, w, pr, B, torch, world, barrier):
     tensors = dict(h)
     tensors.update(dv)
     step = B.make_host_step(scal, head, pr.q_lut, tensors)
-    h2d = sum(h[k].numel() * h[k].element_size() for k in ("h_hidden", "h_src_tokens", "h_lengths", "h_src_tok_off",
-                                                           "h_rewards"))
-    d2h = sum(h[k].numel() * h[k].element_size() for k in ("h_logp", "h_adv", "h_cu_seqlens", "h_survivor_idx", "h_num"))
+    # bytes the call moves per step: small arrays and token ids, the N hidden rows at the detection length, then only
+    # the survivors' hidden rows (uploaded straight into their packed positions); results: logp[T] + per-rollout arrays
+    S_now, T_now = pr.counts()
+    row_bytes = w.d * 2
+    h2d = sum(h[k].numel() * h[k].element_size() for k in ("h_src_tokens", "h_lengths", "h_src_tok_off", "h_rewards"))
+    h2d += (N + T_now) * row_bytes
+    d2h = sum(h[k].numel() * h[k].element_size() for k in ("h_adv", "h_cu_seqlens", "h_survivor_idx", "h_num")) + 4 * T_now + N
     n_e2e = max(1, min(args.steps, 5))
     for _ in range(2):
         B.arrol_prune_rebatch_host(pr.ctx, step)

@@ -55,7 +55,8 @@ int arrol_version(void);                    /* major*10000 + minor*100 + patch *
 const char* arrol_status_string(int status); /* static string, never NULL */
 
 /* Creates a context on CUDA device `device` (made current for the calling thread during the call).
- * Allocates the context's device status word and a small scratch buffer; nothing is allocated later. */
+ * Allocates the context's device status word, a 16 MB scratch buffer, 1 MB of pinned host memory, a second
+ * stream and a few events (used by arrol_prune_rebatch_host); nothing is allocated later. */
 int arrol_create(arrol_ctx** out, int device);
 int arrol_destroy(arrol_ctx* ctx);
 
@@ -243,13 +244,18 @@ int arrol_rank_vote(arrol_ctx* ctx, const float* score, const int32_t* answer, i
                     int32_t* winner, float* winner_weight, void* stream);
 
 /* ---- Whole step from host buffers (Algorithm 1, frontend lines "filter ... rebatch ... log-probs on R'") --
- * Convenience call for callers whose per-step data lives in host memory: copies the step's inputs to the device
- * staging buffers, runs arrol_score_partial -> arrol_select -> arrol_compact -> arrol_token_logprob on `stream`,
- * copies the results back and waits for the stream.  Synchronous; allocates nothing.
+ * Convenience call for callers whose per-step data lives in host memory.  Only what the step needs is uploaded:
+ * the small per-rollout arrays and token ids, the N hidden rows at the detection length (each to its own place in
+ * d_hidden, for the head), and - once arrol_score_partial and arrol_select have produced the keep mask, which is
+ * read back to plan the copies - the survivors' hidden rows, copied straight into their packed positions in
+ * d_dst_rows.  arrol_compact then produces the scan, advantages and packed token ids, and arrol_token_logprob runs
+ * per chunk of tokens as soon as the chunk's rows have landed (uploads on the context's second stream overlap the
+ * tensor-core work).  Results are copied back and the stream is synchronised: the call is synchronous (one
+ * synchronisation in the middle, one at the end) and allocates no device memory.
  * The quality head reads, for rollout i, source row src_tok_off[i] + cutoff - 1 (its hidden state at the
- * detection length); the same source rows are the payload that is compacted and fed to the lm_head.
- * Pointers prefixed h_ are HOST pointers (pinned memory gives full copy speed), d_ are DEVICE buffers provided by
- * the caller with at least the stated sizes.  Model state (head, calib, W_vocab) is device-resident. */
+ * detection length).  Pointers prefixed h_ are HOST pointers (pinned memory gives full copy speed and real overlap),
+ * d_ are DEVICE buffers provided by the caller with at least the stated sizes.  Model state (head, calib, W_vocab)
+ * is device-resident.  P*G <= 1,048,576.  After the call only the scored rows of d_hidden are defined. */
 typedef struct arrol_host_step {
     int32_t P, G, K, cutoff;       /* prompts, group size, survivors per group, detection length (>= 1)         */
     int32_t d, V;                  /* hidden width, vocabulary                                                  */

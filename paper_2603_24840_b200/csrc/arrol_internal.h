@@ -5,6 +5,9 @@
 
 #include "arrol.h"
 
+constexpr int ARROL_COPY_EVENTS = 64;
+constexpr int ARROL_MAX_HOST_N = 1 << 20;   // rollouts per arrol_prune_rebatch_host call
+
 struct arrol_ctx {
     int device;
     int sm_count;
@@ -13,6 +16,9 @@ struct arrol_ctx {
     float* d_scratch;          // MLP-head partial sums: [ARROL_SCRATCH_FLOATS]
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
     unsigned long long launches;   // kernels launched through this context (host-side count)
+    cudaStream_t copy_stream;      // second stream of the host-buffer step: uploads overlap the log-prob kernel
+    cudaEvent_t copy_events[ARROL_COPY_EVENTS];
+    uint8_t* h_keep;               // pinned, ARROL_MAX_HOST_N bytes: the keep mask read back by the host-buffer step
 };
 
 constexpr int ARROL_MAX_MLP_N = 65536;       // rollouts per arrol_score_partial call with an MLP head

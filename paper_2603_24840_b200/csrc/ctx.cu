@@ -44,10 +44,17 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->d_scratch = nullptr;
     ctx->encode_tiled = nullptr;
     ctx->launches = 0;
+    ctx->copy_stream = nullptr;
+    ctx->h_keep = nullptr;
+    for (int i = 0; i < ARROL_COPY_EVENTS; ++i) ctx->copy_events[i] = nullptr;
     bool ok = cudaMalloc(&ctx->d_status, 256) == cudaSuccess &&
               cudaMemset(ctx->d_status, 0, 256) == cudaSuccess &&
               cudaMallocHost(&ctx->h_status, 64) == cudaSuccess &&
-              cudaMalloc(&ctx->d_scratch, ARROL_SCRATCH_FLOATS * sizeof(float)) == cudaSuccess;
+              cudaMalloc(&ctx->d_scratch, ARROL_SCRATCH_FLOATS * sizeof(float)) == cudaSuccess &&
+              cudaMallocHost(&ctx->h_keep, ARROL_MAX_HOST_N) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < ARROL_COPY_EVENTS; ++i)
+        ok = cudaEventCreateWithFlags(&ctx->copy_events[i], cudaEventDisableTiming) == cudaSuccess;
     if (ok) {
         cudaDriverEntryPointQueryResult qres;
         void* fn = nullptr;
@@ -70,6 +77,10 @@ extern "C" int arrol_destroy(arrol_ctx* ctx) {
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
     if (ctx->h_status) (void)cudaFreeHost(ctx->h_status);
     if (ctx->d_scratch) (void)cudaFree(ctx->d_scratch);
+    if (ctx->h_keep) (void)cudaFreeHost(ctx->h_keep);
+    for (int i = 0; i < ARROL_COPY_EVENTS; ++i)
+        if (ctx->copy_events[i]) (void)cudaEventDestroy(ctx->copy_events[i]);
+    if (ctx->copy_stream) (void)cudaStreamDestroy(ctx->copy_stream);
     delete ctx;
     return ARROL_OK;
 }
