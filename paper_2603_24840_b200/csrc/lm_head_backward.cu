@@ -6,12 +6,13 @@
 //
 // The tokens are processed in chunks of TC rows.  Per chunk, three tensor-core kernels with the same
 // TMA -> shared memory -> tcgen05.mma -> tensor memory pipeline as the forward kernel:
-//   dz_kernel      recomputes the chunk's logits tile by tile and turns each accumulator tile into dz (bf16),
-//                  written both as dZ [TC, V] and transposed as dZt [V, TC]
-//   gemm_nt_kernel dH[chunk] = dZ . Wt^T        (M = TC, N = d, K = V;  Wt = W^T, transposed once per call)
-//   gemm_nt_kernel dW       += dZt . Ht^T       (M = V,  N = d, K = TC; Ht = chunk of H transposed)
-// so every contraction is of the K-major x K-major form the forward kernel uses.  The T x V matrix exists only one
-// chunk at a time, in the workspace.
+//   dz_kernel     recomputes the chunk's logits tile by tile and turns each accumulator tile into dz (bf16),
+//                 written once as dZ [TC, V]
+//   gemm_kernel   dH[chunk] = dZ . W       A = dZ K-major (K = V contiguous), B = W MN-major (N = d contiguous)
+//   gemm_kernel   dW       += dZ^T . H     A = dZ MN-major (M = V contiguous), B = H chunk MN-major
+// The MN-major operands are read by the tensor core straight from their row-major storage (transpose bits in the
+// instruction descriptor, MN-major shared-memory descriptors), so nothing is transposed in memory and the T x V
+// matrix exists only one chunk at a time, once, in the workspace.
 #include "arrol_internal.h"
 #include "tc_common.cuh"
 
@@ -22,6 +23,7 @@ constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
 constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int MN_BLOCK_BYTES = BK * 128;   // one 64-element MN block of an MN-major stage: BK rows of 128 bytes
 constexpr int TMEM_COLS = 512;
 constexpr int NUM_THREADS = 192;
 constexpr int EPI_WARPS = 4;
@@ -84,9 +86,11 @@ __device__ __forceinline__ void pipe_teardown(const PipeSmem& ps, uint32_t tmem_
     }
 }
 
-// Producer role (one thread): for every work item, for every K step, one A tile (row coordinate ay) and one
-// B tile (row coordinate by).  `coords(item, ay, by)` returns false when the item list is exhausted.
-template <typename Coords>
+// Producer role (one thread).  For every accumulator tile `coords(it, a_mn0, b_mn0)` gives the operands' MN
+// origins (it returns false when the tile list is exhausted); for every K step the stage receives
+//   K-major operand:  one box  [MN rows x 64 K columns]           at (x = k, y = mn0)
+//   MN-major operand: MN/64 boxes [64 K rows x 64 MN columns]     at (x = mn0 + 64 b, y = k), BK*128 bytes apart.
+template <bool A_MN, bool B_MN, typename Coords>
 __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensorMap* ma, const CUtensorMap* mb,
                                               int k_steps, Coords coords) {
     uint32_t stage = 0, phase = 0, issued = 0;
@@ -96,8 +100,20 @@ __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensor
         for (int ks = 0; ks < k_steps; ++ks) {
             if (!mbar_wait(&ps.empty[stage], phase ^ 1u, ps.abort_flag)) { ok = false; break; }
             mbar_expect_tx(&ps.full[stage], STAGE_BYTES);
-            tma_load_2d(ps.stage_a + (size_t)stage * A_STAGE_BYTES, ma, ks * BK, ay, &ps.full[stage]);
-            tma_load_2d(ps.stage_b + (size_t)stage * B_STAGE_BYTES, mb, ks * BK, by, &ps.full[stage]);
+            uint8_t* sa = ps.stage_a + (size_t)stage * A_STAGE_BYTES;
+            uint8_t* sb = ps.stage_b + (size_t)stage * B_STAGE_BYTES;
+            if constexpr (A_MN) {
+#pragma unroll
+                for (int b = 0; b < BM / 64; ++b) tma_load_2d(sa + b * MN_BLOCK_BYTES, ma, ay + 64 * b, ks * BK, &ps.full[stage]);
+            } else {
+                tma_load_2d(sa, ma, ks * BK, ay, &ps.full[stage]);
+            }
+            if constexpr (B_MN) {
+#pragma unroll
+                for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * MN_BLOCK_BYTES, mb, by + 64 * b, ks * BK, &ps.full[stage]);
+            } else {
+                tma_load_2d(sb, mb, ks * BK, by, &ps.full[stage]);
+            }
             ++issued;
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -114,8 +130,13 @@ __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensor
 }
 
 // MMA role (one thread): n_items accumulator tiles of k_steps K steps each, alternating the two accumulators.
+// Inside a stage the four K = 16 slices are 32 bytes apart for a K-major operand (columns of the swizzled row) and
+// 16 rows = 2048 bytes apart for an MN-major one.
+template <bool A_MN, bool B_MN>
 __device__ __forceinline__ void mma_loop(const PipeSmem& ps, uint32_t tmem_base, int64_t n_items, int k_steps) {
-    constexpr uint32_t idesc = make_idesc(BM, BN);
+    constexpr uint32_t idesc = make_idesc(BM, BN, A_MN, B_MN);
+    constexpr uint64_t a_step = A_MN ? (UMMA_K * 128) >> 4 : (UMMA_K * 2) >> 4;
+    constexpr uint64_t b_step = B_MN ? (UMMA_K * 128) >> 4 : (UMMA_K * 2) >> 4;
     uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
     bool ok = true;
     for (int64_t it = 0; it < n_items && ok; ++it) {
@@ -125,12 +146,13 @@ __device__ __forceinline__ void mma_loop(const PipeSmem& ps, uint32_t tmem_base,
         for (int ks = 0; ks < k_steps; ++ks) {
             if (!mbar_wait(&ps.full[stage], phase, ps.abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
-            const uint64_t a_desc = make_smem_desc(smem_u32(ps.stage_a + (size_t)stage * A_STAGE_BYTES));
-            const uint64_t b_desc = make_smem_desc(smem_u32(ps.stage_b + (size_t)stage * B_STAGE_BYTES));
+            const uint32_t sa = smem_u32(ps.stage_a + (size_t)stage * A_STAGE_BYTES);
+            const uint32_t sb = smem_u32(ps.stage_b + (size_t)stage * B_STAGE_BYTES);
+            const uint64_t a_desc = A_MN ? make_smem_desc_mn(sa, BK) : make_smem_desc(sa);
+            const uint64_t b_desc = B_MN ? make_smem_desc_mn(sb, BK) : make_smem_desc(sb);
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k)
-                tcgen05_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                 (ks | k) != 0 ? 1u : 0u);
+                tcgen05_mma_bf16(d_tmem, a_desc + a_step * k, b_desc + b_step * k, idesc, (ks | k) != 0 ? 1u : 0u);
             tcgen05_commit(&ps.empty[stage]);
             if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -162,7 +184,6 @@ struct DzParams {
     int splits, chunks_per_split;
     float scale2, inv_temp;
     __nv_bfloat16* dZ;        // [TC, ldz]
-    __nv_bfloat16* dZt;       // [V, TC]
     uint32_t* d_status;
 };
 
@@ -191,7 +212,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
             int64_t item = blockIdx.x;
             int m_tile = 0, c = 0, c1 = 0;
             bool have = false;
-            producer_loop(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
+            producer_loop<false, false>(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
                 while (!have || c >= c1) {
                     if (have) item += gridDim.x;
                     if (item >= items) return false;
@@ -212,7 +233,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                 item_range(item, m_tile, c0, c1);
                 n_tiles += max(c1 - c0, 0);
             }
-            mma_loop(ps, tmem_base, n_tiles, k_steps);
+            mma_loop<false, false>(ps, tmem_base, n_tiles, k_steps);
         }
     } else {
         const int quarter = warp & 3;
@@ -261,7 +282,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                         packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
                     }
                     const int n_valid = min(32, p.V - pc0);
-                    if (n_valid == 32 && (p.ldz & 7) == 0) {
+                    if (n_valid == 32) {
                         uint4* dst = reinterpret_cast<uint4*>(zrow + pc0);
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4)
@@ -275,15 +296,6 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                             }
                         }
                     }
-                    // transposed copy: for a fixed vocabulary row the 32 lanes write 32 consecutive tokens (64 bytes)
-                    uint16_t* zt = reinterpret_cast<uint16_t*>(p.dZt) + (int64_t)pc0 * TC + row_in_chunk;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (j < n_valid) {
-                            const uint32_t w = packed[j >> 1];
-                            zt[(int64_t)j * TC] = (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu));
-                        }
-                    }
                 }
                 tcgen05_fence_before();
                 __syncwarp();
@@ -295,32 +307,37 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
     pipe_teardown(ps, tmem_base, p.d_status);
 }
 
-// ---- generic C[M,N] (+)= A[M,K] B[N,K]^T, bf16 operands K-major, fp32 result -------------------------------------
+// ---- C[M,N] (+)= op(A) op(B): bf16 operands in either orientation, fp32 result ------------------------------------
+//   A_MN = false: A stored [M, K] row-major;  A_MN = true: A stored [K, M] row-major (used as its transpose)
+//   B_MN = false: B stored [N, K] row-major;  B_MN = true: B stored [K, N] row-major
 struct GemmParams {
     int M, N, K;
     float* C;
     int64_t ldc;
-    int accumulate;           // 1: C += A B^T, 0: C = A B^T
+    int accumulate;           // 1: C += ..., 0: C = ...
+    int k_is_tokens;          // 1: K counts the chunk's tokens: only the live ones (T - t0) are contracted
     const int64_t* d_T;       // the launch is skipped when t0 >= live tokens
     int64_t T_max, t0;
     uint32_t* d_status;
 };
 
+template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_nt_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const GemmParams p) {
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const PipeSmem ps = carve_smem(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (p.t0 >= live_tokens(p.d_T, p.T_max)) return;
+    const int64_t T_live = live_tokens(p.d_T, p.T_max);
+    if (p.t0 >= T_live) return;
     const int m_tiles = (p.M + BM - 1) / BM, n_tiles = (p.N + BN - 1) / BN;
     const int64_t items = (int64_t)m_tiles * n_tiles;
-    const int k_steps = (p.K + BK - 1) / BK;
+    const int K = p.k_is_tokens ? (int)min((int64_t)p.K, T_live - p.t0) : p.K;
+    const int k_steps = (K + BK - 1) / BK;
     const uint32_t tmem_base = pipe_setup(ps, &map_a, &map_b);
 
     if (warp == 0) {
         if (lane == 0) {
-            producer_loop(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
+            producer_loop<A_MN, B_MN>(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
                 const int64_t item = blockIdx.x + it * gridDim.x;
                 if (item >= items) return false;
                 ay = (int)(item / n_tiles) * BM;       // consecutive blocks share the A panel, walk the B panels
@@ -331,7 +348,7 @@ gemm_nt_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         if (lane == 0) {
             const int64_t mine = items > blockIdx.x ? (items - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-            mma_loop(ps, tmem_base, mine, k_steps);
+            mma_loop<A_MN, B_MN>(ps, tmem_base, mine, k_steps);
         }
     } else {
         const int quarter = warp & 3;
@@ -380,53 +397,16 @@ gemm_nt_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     pipe_teardown(ps, tmem_base, p.d_status);
 }
 
-// ---- bf16 transpose: dst[c, r] = src[r, c] for r < rows_live, zero for rows_live <= r < rows -------------------
-__global__ void transpose_bf16_kernel(const uint16_t* __restrict__ src, int64_t ld_src, int64_t rows, int64_t cols,
-                                      uint16_t* __restrict__ dst, int64_t ld_dst, const int64_t* d_T, int64_t T_max,
-                                      int64_t t0, int use_live) {
-    __shared__ uint16_t tile[64][66];
-    int64_t rows_live = rows;
-    if (use_live) {
-        const int64_t T = live_tokens(d_T, T_max);
-        if (t0 >= T) return;
-        rows_live = min(rows, T - t0);
-    }
-    const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;
-    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-        const int64_t r = r0 + i, c = c0 + threadIdx.x * 2;
-        uint16_t a = 0, b = 0;
-        if (r < rows_live) {
-            if (c < cols) a = src[r * ld_src + c];
-            if (c + 1 < cols) b = src[r * ld_src + c + 1];
-        }
-        tile[i][threadIdx.x * 2] = a;
-        tile[i][threadIdx.x * 2 + 1] = b;
-    }
-    __syncthreads();
-    for (int i = threadIdx.y; i < 64; i += blockDim.y) {
-        const int64_t c = c0 + i, r = r0 + threadIdx.x * 2;
-        if (c < cols) {
-            if (r < rows) dst[c * ld_dst + r] = tile[threadIdx.x * 2][i];
-            if (r + 1 < rows) dst[c * ld_dst + r + 1] = tile[threadIdx.x * 2 + 1][i];
-        }
-    }
-}
-
 struct BackwardLayout {
     int64_t ldz;       // V rounded up to 8
-    size_t wt, dz, dzt, ht, total;
+    size_t dz, total;
 };
 
-BackwardLayout backward_layout(int d, int V) {
+BackwardLayout backward_layout(int V) {
     BackwardLayout L;
     L.ldz = ((int64_t)V + 7) & ~(int64_t)7;
-    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
-    size_t o = 0;
-    L.wt = o; o = up(o + (size_t)d * L.ldz * 2);
-    L.dz = o; o = up(o + (size_t)TC * L.ldz * 2);
-    L.dzt = o; o = up(o + (size_t)V * TC * 2);
-    L.ht = o; o = up(o + (size_t)d * TC * 2);
-    L.total = o;
+    L.dz = 0;
+    L.total = (((size_t)TC * L.ldz * 2) + 255) & ~(size_t)255;
     return L;
 }
 
@@ -434,7 +414,7 @@ BackwardLayout backward_layout(int d, int V) {
 
 extern "C" size_t arrol_lm_head_backward_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
     if (!ctx || T_max <= 0 || d <= 0 || V <= 0) return 0;
-    return backward_layout(d, V).total;
+    return backward_layout(V).total;
 }
 
 extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
@@ -453,31 +433,22 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     if (!hidden || !W_vocab || !targets || !grad_logp || !lse || !dH) return ARROL_ERR_INVALID_ARG;
     if (!arrol_aligned(hidden, 16) || !arrol_aligned(W_vocab, 16) || !arrol_aligned(dH, 16) || !arrol_aligned(dW, 16))
         return ARROL_ERR_INVALID_ARG;
-    const BackwardLayout L = backward_layout(d, V);
+    const BackwardLayout L = backward_layout(V);
     if (!workspace || workspace_bytes < L.total || !arrol_aligned(workspace, 256)) return ARROL_ERR_WORKSPACE;
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    uint16_t* Wt = reinterpret_cast<uint16_t*>(ws + L.wt);
-    __nv_bfloat16* dZ = reinterpret_cast<__nv_bfloat16*>(ws + L.dz);
-    __nv_bfloat16* dZt = reinterpret_cast<__nv_bfloat16*>(ws + L.dzt);
-    uint16_t* Ht = reinterpret_cast<uint16_t*>(ws + L.ht);
+    __nv_bfloat16* dZ = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + L.dz);
 
     ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_nt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
 
-    // W^T once per call: [V, d] -> [d, ldz]
-    {
-        dim3 grid((unsigned)((d + 63) / 64), (unsigned)((V + 63) / 64)), block(32, 8);
-        transpose_bf16_kernel<<<grid, block, 0, s>>>(static_cast<const uint16_t*>(W_vocab), d, V, d, Wt, L.ldz, nullptr,
-                                                     0, 0, 0);
-        ctx->launches += 1;
-    }
-    CUtensorMap map_h, map_w, map_dz, map_wt, map_dzt, map_ht;
-    if (make_map(ctx, &map_h, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map_ld(ctx, &map_dz, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map_ld(ctx, &map_wt, Wt, (uint64_t)d, (uint64_t)V, (uint64_t)L.ldz, BN) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map_ld(ctx, &map_dzt, dZt, (uint64_t)V, TC, TC, BM) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map_ld(ctx, &map_ht, Ht, (uint64_t)d, TC, TC, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+    // tensor maps: K-major operands are fetched as [MN rows x 64 K columns] boxes, MN-major ones as [64 K rows x 64 MN
+    // columns] boxes of the same row-major storage
+    CUtensorMap map_h_k, map_w_k, map_dz_k, map_w_mn, map_dz_mn, map_h_mn;
+    if (make_map(ctx, &map_h_k, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map(ctx, &map_w_k, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_dz_k, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_dz_mn, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BK) != ARROL_OK) return ARROL_ERR_CUDA;
 
     const int total_chunks = (V + BN - 1) / BN;
     int splits = 1;
@@ -486,34 +457,34 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     splits = (total_chunks + chunks_per_split - 1) / chunks_per_split;
 
     for (int64_t t0 = 0; t0 < T_max; t0 += TC) {
+        const int64_t rows = (T_max - t0) < TC ? (T_max - t0) : (int64_t)TC;
+        // the chunk of hidden as an MN-major B operand: [rows (K), d (N)]; rows past T_max read as zero
+        if (make_map(ctx, &map_h_mn, static_cast<const uint8_t*>(hidden) + (size_t)t0 * d * 2, (uint64_t)rows, (uint64_t)d,
+                     BK) != ARROL_OK)
+            return ARROL_ERR_CUDA;
+
         DzParams zp;
         zp.targets = targets; zp.grad_logp = grad_logp; zp.lse = lse; zp.d_T = d_T; zp.T_max = T_max; zp.t0 = t0;
         zp.d = d; zp.V = V; zp.ldz = L.ldz; zp.splits = splits; zp.chunks_per_split = chunks_per_split;
         zp.scale2 = inv_temperature * 1.44269504088896340736f; zp.inv_temp = inv_temperature;
-        zp.dZ = dZ; zp.dZt = dZt; zp.d_status = ctx->d_status;
+        zp.dZ = dZ; zp.d_status = ctx->d_status;
         int64_t grid = (int64_t)(TC / BM) * splits;
         if (grid > ctx->sm_count) grid = ctx->sm_count;
-        dz_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, zp);
+        dz_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h_k, map_w_k, zp);
 
-        const int64_t rows = (T_max - t0) < TC ? (T_max - t0) : (int64_t)TC;
-        {   // chunk of H transposed, columns past the live tokens zeroed: [rows, d] -> [d, TC]
-            dim3 tg((unsigned)((d + 63) / 64), (unsigned)(TC / 64)), block(32, 8);
-            transpose_bf16_kernel<<<tg, block, 0, s>>>(static_cast<const uint16_t*>(hidden) + t0 * d, d, TC, d, Ht, TC,
-                                                       d_T, T_max, t0, 1);
-        }
-        GemmParams gh;
-        gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0;
+        GemmParams gh;    // dH[chunk] = dZ . W
+        gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0; gh.k_is_tokens = 0;
         gh.d_T = d_T; gh.T_max = T_max; gh.t0 = t0; gh.d_status = ctx->d_status;
-        int64_t gh_items = (int64_t)((rows + BM - 1) / BM) * ((d + BN - 1) / BN);
-        gemm_nt_kernel<<<(unsigned)(gh_items < ctx->sm_count ? gh_items : ctx->sm_count), NUM_THREADS, SMEM_BYTES, s>>>(
-            map_dz, map_wt, gh);
-        GemmParams gw;
-        gw.M = V; gw.N = d; gw.K = TC; gw.C = dW; gw.ldc = d; gw.accumulate = 1;
+        const int64_t gh_items = (int64_t)((rows + BM - 1) / BM) * ((d + BN - 1) / BN);
+        gemm_kernel<false, true><<<(unsigned)(gh_items < ctx->sm_count ? gh_items : ctx->sm_count), NUM_THREADS,
+                                   SMEM_BYTES, s>>>(map_dz_k, map_w_mn, gh);
+        GemmParams gw;    // dW += dZ^T . H[chunk]
+        gw.M = V; gw.N = d; gw.K = (int)rows; gw.C = dW; gw.ldc = d; gw.accumulate = 1; gw.k_is_tokens = 1;
         gw.d_T = d_T; gw.T_max = T_max; gw.t0 = t0; gw.d_status = ctx->d_status;
-        int64_t gw_items = (int64_t)((V + BM - 1) / BM) * ((d + BN - 1) / BN);
-        gemm_nt_kernel<<<(unsigned)(gw_items < ctx->sm_count ? gw_items : ctx->sm_count), NUM_THREADS, SMEM_BYTES, s>>>(
-            map_dzt, map_ht, gw);
-        ctx->launches += 4;
+        const int64_t gw_items = (int64_t)((V + BM - 1) / BM) * ((d + BN - 1) / BN);
+        gemm_kernel<true, true><<<(unsigned)(gw_items < ctx->sm_count ? gw_items : ctx->sm_count), NUM_THREADS,
+                                  SMEM_BYTES, s>>>(map_dz_mn, map_h_mn, gw);
+        ctx->launches += 3;
         ARROL_CUDA_OK(cudaGetLastError());
     }
     return ARROL_OK;
