@@ -90,7 +90,7 @@ __device__ __forceinline__ void pipe_teardown(const PipeSmem& ps, uint32_t tmem_
 // origins (it returns false when the tile list is exhausted); for every K step the stage receives
 //   K-major operand:  one box  [MN rows x 64 K columns]           at (x = k, y = mn0)
 //   MN-major operand: MN/64 boxes [64 K rows x 64 MN columns]     at (x = mn0 + 64 b, y = k), BK*128 bytes apart.
-template <bool A_MN, bool B_MN, typename Coords>
+template <bool A_MN, bool B_MN, int PF, typename Coords>
 __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensorMap* ma, const CUtensorMap* mb,
                                               int k_steps, Coords coords) {
     uint32_t stage = 0, phase = 0, issued = 0;
@@ -99,6 +99,23 @@ __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensor
     for (int64_t it = 0; ok && coords(it, ay, by); ++it) {
         for (int ks = 0; ks < k_steps; ++ks) {
             if (!mbar_wait(&ps.empty[stage], phase ^ 1u, ps.abort_flag)) { ok = false; break; }
+            if constexpr (PF > 0) {   // pull the tiles PF steps ahead into L2 (operands that stream from HBM)
+                const int kp = (ks + PF) * BK;
+                if (ks + PF < k_steps) {
+                    if constexpr (A_MN) {
+#pragma unroll
+                        for (int b = 0; b < BM / 64; ++b) tma_prefetch_l2_2d(ma, ay + 64 * b, kp);
+                    } else {
+                        tma_prefetch_l2_2d(ma, kp, ay);
+                    }
+                    if constexpr (B_MN) {
+#pragma unroll
+                        for (int b = 0; b < BN / 64; ++b) tma_prefetch_l2_2d(mb, by + 64 * b, kp);
+                    } else {
+                        tma_prefetch_l2_2d(mb, kp, by);
+                    }
+                }
+            }
             mbar_expect_tx(&ps.full[stage], STAGE_BYTES);
             uint8_t* sa = ps.stage_a + (size_t)stage * A_STAGE_BYTES;
             uint8_t* sb = ps.stage_b + (size_t)stage * B_STAGE_BYTES;
@@ -212,7 +229,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
             int64_t item = blockIdx.x;
             int m_tile = 0, c = 0, c1 = 0;
             bool have = false;
-            producer_loop<false, false>(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
+            producer_loop<false, false, 0>(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
                 while (!have || c >= c1) {
                     if (have) item += gridDim.x;
                     if (item >= items) return false;
@@ -263,18 +280,18 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                 ok = __all_sync(0xffffffffu, ok) != 0;
                 if (!ok) break;
                 tcgen05_fence_after();
-#pragma unroll 1
-                for (int piece = 0; piece < BN / 32; ++piece) {
+                // Two register buffers: the tensor-memory load of piece i + 1 is in flight while piece i is turned
+                // into dz and stored.
+                const uint32_t tacc = tmem_base + lane_addr + acc * BN;
+                auto emit = [&](const uint32_t (&raw)[32], int piece) {
                     const int pc0 = c * BN + piece * 32;
-                    if (pc0 >= p.V) break;
-                    float v[32];
-                    tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
+                    if (pc0 >= p.V) return;
                     uint32_t packed[16];
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
                         // dz = coef ([v = y] - 2^(z log2e - lse log2e)); coef = 0 for rows that carry no gradient
-                        float d0 = -coef * ex2_approx(fmaf(v[j], p.scale2, -lse2));
-                        float d1 = -coef * ex2_approx(fmaf(v[j + 1], p.scale2, -lse2));
+                        float d0 = -coef * ex2_approx(fmaf(__uint_as_float(raw[j]), p.scale2, -lse2));
+                        float d1 = -coef * ex2_approx(fmaf(__uint_as_float(raw[j + 1]), p.scale2, -lse2));
                         if (pc0 + j == y) d0 += coef;
                         if (pc0 + j + 1 == y) d1 += coef;
                         if (coef == 0.f) { d0 = 0.f; d1 = 0.f; }      // also guards 0 * inf from stale lse values
@@ -296,6 +313,17 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                             }
                         }
                     }
+                };
+                uint32_t ra[32], rb[32];
+                tcgen05_ld_32x32_issue(tacc, ra);
+#pragma unroll 1
+                for (int piece = 0; piece < BN / 32; piece += 2) {
+                    tcgen05_ld_wait(ra);
+                    tcgen05_ld_32x32_issue(tacc + (piece + 1) * 32, rb);
+                    emit(ra, piece);
+                    tcgen05_ld_wait(rb);
+                    if (piece + 2 < BN / 32) tcgen05_ld_32x32_issue(tacc + (piece + 2) * 32, ra);
+                    emit(rb, piece + 1);
                 }
                 tcgen05_fence_before();
                 __syncwarp();
@@ -337,7 +365,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
     if (warp == 0) {
         if (lane == 0) {
-            producer_loop<A_MN, B_MN>(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
+            producer_loop<A_MN, B_MN, 0>(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
                 const int64_t item = blockIdx.x + it * gridDim.x;
                 if (item >= items) return false;
                 ay = (int)(item / n_tiles) * BM;       // consecutive blocks share the A panel, walk the B panels
