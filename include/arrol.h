@@ -217,6 +217,22 @@ int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_voc
                            int32_t V, float inv_temperature, float* dH, float* dW, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* ---- Trace confidence (Section 3 "Trace Confidence") ---------------------------------------------------------
+ * arrol_token_logprob_conf: arrol_token_logprob with one more output from the same launch, the token confidence
+ *     token_conf[t] = H_t = - sum_{v < V} log P_t(v) = V lse[t] - sum_v z_{t,v}     (float [T_max], rows t < T)
+ *   accumulated in the same epilogue (one more add per logit).  All other arguments as arrol_token_logprob.
+ * arrol_trace_confidence: per packed trace s < S (S read from d_num = {S, T}; bounds from cu_seqlens):
+ *     mode 0: trace_conf[s] = mean of token_conf over the trace;
+ *     mode 1: trace_conf[s] = minimum over the trace of the mean of token_conf over a sliding window of `window`
+ *             tokens (a trace shorter than the window has one window, the whole trace).
+ *   An empty trace gives 0.  trace_conf float [S_max].  fp64 accumulation. */
+int arrol_token_logprob_conf(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                             int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
+                             float* logp, float* lse, float* token_conf, void* workspace, size_t workspace_bytes,
+                             void* stream);
+int arrol_trace_confidence(arrol_ctx* ctx, const float* token_conf, const int64_t* cu_seqlens, const int64_t* d_num,
+                           int32_t S_max, int32_t window, int32_t mode, float* trace_conf, void* stream);
+
 /* ---- Quality-head training step (Section 4.2; Section 4.3 (iii)) ------------------------------------------
  * Cross-entropy of the head's logit against the rollout's final reward, gradients into the head only:
  *     y_i = rewards[i] > 0.5;  over the n rollouts with mask[i] != 0 (all when mask is NULL; e.g. the survivors, the

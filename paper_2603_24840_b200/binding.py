@@ -25,7 +25,7 @@ EXPORTS = [
     "arrol_calib_state_bytes", "arrol_calib_layout", "arrol_calib_init", "arrol_calib_update", "arrol_calib_q_lut",
     "arrol_calib_delta", "arrol_select_stochastic",
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
-    "arrol_head_grad_workspace", "arrol_head_grad",
+    "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
 ]
 
 

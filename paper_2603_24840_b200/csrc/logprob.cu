@@ -31,8 +31,8 @@ constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 
-struct PartialLse {   // per (split, token): running maximum and sum in the base-2 domain, target logit
-    float m2, l, zy2, pad;
+struct PartialLse {   // per (split, token): running maximum and sum in the base-2 domain, target logit,
+    float m2, l, zy2, pad;   // pad: sum of the raw accumulators of the split (only when the confidence is asked for)
 };
 
 struct LogprobParams {
@@ -45,10 +45,13 @@ struct LogprobParams {
     float scale2;          // inv_temperature * log2(e)
     float* logp;
     float* lse;
+    float* conf;           // token confidence H_t = -sum_v log P_t(v) = V lse - sum_v z_v, or NULL
+    float inv_temp;
     PartialLse* partial;   // [splits][T_max] when splits > 1
     uint32_t* d_status;
 };
 
+template <bool CONF>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
                      const LogprobParams p) {
@@ -179,7 +182,7 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
             const int c1 = min(c0 + p.chunks_per_split, total_chunks);
             const int64_t t = (int64_t)m_tile * BM + row_in_tile;
             const int y = (t < T) ? p.targets[t] : -1;
-            float m2 = -INFINITY, l = 0.f, zy2 = -INFINITY;
+            float m2 = -INFINITY, l = 0.f, zy2 = -INFINITY, sumz = 0.f;
             for (int c = c0; c < c1 && ok; ++c) {
                 ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
                 ok = __all_sync(0xffffffffu, ok) != 0;     // keep the warp converged for the aligned tensor-memory loads
@@ -192,6 +195,12 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                     if (pc0 >= p.V) break;                  // columns past the vocabulary (zero-filled by TMA)
                     float v[32];
                     tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
+                    if constexpr (CONF) {                   // sum of the valid logits of the piece (before masking)
+                        float ps = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) ps += (pc0 + j < p.V) ? v[j] : 0.f;
+                        sumz += ps;
+                    }
                     if (pc0 + 32 > p.V) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) if (pc0 + j >= p.V) v[j] = -INFINITY;
@@ -227,9 +236,10 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                     }
                     p.logp[t] = out;
                     if (p.lse) p.lse[t] = lse2 * ln2;
+                    if constexpr (CONF) p.conf[t] = (float)p.V * (lse2 * ln2) - sumz * p.inv_temp;
                 } else {
                     PartialLse pr;
-                    pr.m2 = m2; pr.l = l; pr.zy2 = zy2; pr.pad = 0.f;
+                    pr.m2 = m2; pr.l = l; pr.zy2 = zy2; pr.pad = sumz;
                     *reinterpret_cast<float4*>(&p.partial[(int64_t)split * p.T_max + t]) =
                         make_float4(pr.m2, pr.l, pr.zy2, pr.pad);
                 }
@@ -249,7 +259,8 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
 // Merge of the per-split (max, sum, target logit) triples: M = max m_s, L = sum l_s 2^(m_s - M).
 __global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, const int32_t* __restrict__ targets,
                                       const int64_t* __restrict__ d_T, int64_t T_max, int V, int splits,
-                                      float* __restrict__ logp, float* __restrict__ lse, uint32_t* d_status) {
+                                      float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ conf,
+                                      float inv_temp, uint32_t* d_status) {
     int64_t T = T_max;
     if (d_T) { const int64_t t = *d_T; T = t < 0 ? 0 : (t < T ? t : T); }
     for (int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
@@ -259,10 +270,11 @@ __global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, co
             M = fmaxf(M, pr.x);
             zy2 = fmaxf(zy2, pr.z);          // exactly one split holds the target column; the others hold -inf
         }
-        float L = 0.f;
+        float L = 0.f, sumz = 0.f;
         for (int s = 0; s < splits; ++s) {
             const float4 pr = *reinterpret_cast<const float4*>(&partial[(int64_t)s * T_max + t]);
             L += pr.y * exp2f(pr.x - M);
+            sumz += pr.w;
         }
         const float lse2 = M + log2f(L);
         const float ln2 = 0.69314718055994530942f;
@@ -274,6 +286,7 @@ __global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, co
         }
         logp[t] = out;
         if (lse) lse[t] = lse2 * ln2;
+        if (conf) conf[t] = (float)V * (lse2 * ln2) - sumz * inv_temp;
     }
 }
 
@@ -302,10 +315,10 @@ extern "C" size_t arrol_token_logprob_workspace(arrol_ctx* ctx, int64_t T_max, i
     return (size_t)splits * (size_t)T_max * sizeof(PartialLse) + 256;
 }
 
-extern "C" int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
-                                   int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
-                                   float* logp, float* lse, void* workspace, size_t workspace_bytes,
-                                   void* stream) {
+static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                             int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
+                             float* logp, float* lse, float* conf, void* workspace, size_t workspace_bytes,
+                             void* stream) {
     if (!ctx || T_max < 0 || d <= 0 || V <= 0 || !(inv_temperature > 0.f)) return ARROL_ERR_INVALID_ARG;
     if (T_max == 0) return ARROL_OK;
     if (!hidden || !W_vocab || !targets || !logp) return ARROL_ERR_INVALID_ARG;
@@ -336,24 +349,46 @@ extern "C" int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const voi
     p.scale2 = inv_temperature * 1.44269504088896340736f;
     p.logp = logp;
     p.lse = lse;
+    p.conf = conf;
+    p.inv_temp = inv_temperature;
     p.partial = static_cast<PartialLse*>(workspace);
     p.d_status = ctx->d_status;
 
-    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)SMEM_BYTES));
     const int64_t m_tiles = (T_max + BM - 1) / BM;
     int64_t grid = m_tiles * p.splits;
     if (grid > ctx->sm_count) grid = ctx->sm_count;
-    token_logprob_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
+    if (conf) token_logprob_kernel<true><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
+    else token_logprob_kernel<false><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     if (p.splits > 1) {
         int64_t blocks = (T_max + 255) / 256;
         if (blocks > (int64_t)ctx->sm_count * 8) blocks = (int64_t)ctx->sm_count * 8;
         combine_splits_kernel<<<(unsigned)blocks, 256, 0, s>>>(p.partial, targets, d_T, T_max, V, p.splits, logp,
-                                                              lse, ctx->d_status);
+                                                              lse, conf, inv_temperature, ctx->d_status);
         ctx->launches += 1;
         ARROL_CUDA_OK(cudaGetLastError());
     }
     return ARROL_OK;
+}
+
+extern "C" int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                                   int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
+                                   float* logp, float* lse, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+    return run_token_logprob(ctx, hidden, W_vocab, targets, T_max, d_T, d, V, inv_temperature, logp, lse, nullptr,
+                             workspace, workspace_bytes, stream);
+}
+
+extern "C" int arrol_token_logprob_conf(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
+                                        int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
+                                        float* logp, float* lse, float* token_conf, void* workspace,
+                                        size_t workspace_bytes, void* stream) {
+    if (T_max > 0 && !token_conf) return ARROL_ERR_INVALID_ARG;
+    return run_token_logprob(ctx, hidden, W_vocab, targets, T_max, d_T, d, V, inv_temperature, logp, lse, token_conf,
+                             workspace, workspace_bytes, stream);
 }
