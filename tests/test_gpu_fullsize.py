@@ -8,14 +8,16 @@ import torch
 
 import oracle
 from paper_2603_24840_b200 import binding as B
-from paper_2603_24840_b200 import synth
+from paper_2603_24840_b200 import dist_util, synth
 from paper_2603_24840_b200.pipeline import PruneRebatch, host_inputs
 
 pytestmark = pytest.mark.gpu
 
 
-def _fullsize(name, n_logp_rows):
+def _fullsize(name, n_logp_rows, prompt_chunks=1):
     w = synth.WORKLOADS[name]
+    if prompt_chunks > 1:                       # the benchmark runs this workload as chunks of P / prompt_chunks prompts
+        w = dist_util.shard_workload(w, 0, 1, prompt_chunks=prompt_chunks)
     inp = host_inputs(w)                       # big tensors are generated on the device
     pr = PruneRebatch(w, inputs=inp)
     pr.step()
@@ -93,3 +95,11 @@ def test_llama_3_2_1b_shaped():
 
 def test_qwen3_1_7b_shaped():
     _fullsize("qwen3-1.7b", 24)
+
+
+def test_qwen3_4b_shaped():
+    _fullsize("qwen3-4b", 16)
+
+
+def test_qwen3_8b_dapo_shaped_one_prompt_chunk():
+    _fullsize("qwen3-8b-dapo", 16, prompt_chunks=4)
