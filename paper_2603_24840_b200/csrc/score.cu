@@ -113,12 +113,16 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
 // shared memory (two shared buffers, one barrier per chunk).
 constexpr int TM = 64, TH = ARROL_MLP_TH, TK = 32, PAD = 4, MLP_THREADS = 128;
 
-template <typename T>
+// SPLITK = false: the block contracts the whole of d and finishes its tile (bias, GELU, w2 dot) -> partial [h_tiles][N].
+// SPLITK = true:  blockIdx.z picks a K range of k_len columns; the raw partial pre-activations go to
+//                 partial [splits][N][h] and score_mlp_splitk_finish_kernel completes them.  More, shorter blocks:
+//                 this is what fills the SMs when N x h is only a few hundred tiles.
+template <typename T, bool SPLITK>
 __global__ void __launch_bounds__(MLP_THREADS)
 score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index,
                       int N, int d, int h, const T* __restrict__ W1, const T* __restrict__ b1,
-                      const T* __restrict__ w2, float* __restrict__ partial /* [h_tiles][N] */,
-                      float* __restrict__ u_out /* [N][h] pre-activations, or NULL */) {
+                      const T* __restrict__ w2, float* __restrict__ partial,
+                      float* __restrict__ u_out /* [N][h] pre-activations, or NULL */, int k_len) {
     constexpr int VN = Vec16<T>::N;
     constexpr int VPR = TK / VN;                       // 16-byte vectors per tile row per K chunk
     constexpr int NV = TM * VPR / MLP_THREADS;         // vectors per thread per operand per chunk (2 or 4)
@@ -145,17 +149,18 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
         if (m < N) xrow[i] = hidden + (row_index ? row_index[m] : (int64_t)m) * row_stride;
         if (j < h) wrow[i] = W1 + (int64_t)j * d;
     }
+    const int k_end = SPLITK ? min(d, ((int)blockIdx.z + 1) * k_len) : d;
     float xreg[NV][VN], wreg[NV][VN];
     auto fetch = [&](int k0) {
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             const int k = k0 + kofs[i];
-            if (xrow[i] && k < d) Vec16<T>::load(xrow[i] + k, xreg[i]);
+            if (xrow[i] && k < k_end) Vec16<T>::load(xrow[i] + k, xreg[i]);
             else {
 #pragma unroll
                 for (int e = 0; e < VN; ++e) xreg[i][e] = 0.f;
             }
-            if (wrow[i] && k < d) Vec16<T>::load(wrow[i] + k, wreg[i]);
+            if (wrow[i] && k < k_end) Vec16<T>::load(wrow[i] + k, wreg[i]);
             else {
 #pragma unroll
                 for (int e = 0; e < VN; ++e) wreg[i][e] = 0.f;
@@ -178,12 +183,14 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
 
-    fetch(0);
+    const int k_lo = SPLITK ? (int)blockIdx.z * k_len : 0;
+    const int k_hi = SPLITK ? min(d, k_lo + k_len) : d;
+    fetch(k_lo);
     stash(0);
     __syncthreads();
     int buf = 0;
-    for (int k0 = 0; k0 < d; k0 += TK, buf ^= 1) {
-        const bool more = k0 + TK < d;
+    for (int k0 = k_lo; k0 < k_hi; k0 += TK, buf ^= 1) {
+        const bool more = k0 + TK < k_hi;
         if (more) fetch(k0 + TK);
 #pragma unroll
         for (int k = 0; k < TK; ++k) {
@@ -201,6 +208,16 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
         __syncthreads();
     }
 
+    if constexpr (SPLITK) {   // raw partial pre-activations of this K range
+        float* out = partial + (int64_t)blockIdx.z * N * h;
+#pragma unroll
+        for (int a = 0; a < 8; ++a) {
+            const int m = m0 + ty * 8 + a, j = j0 + tx * 4;
+            if (m < N && j < h)     // h % 4 == 0: a float4 never straddles the edge
+                *reinterpret_cast<float4*>(out + (int64_t)m * h + j) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
+        }
+        return;
+    }
     // epilogue: u + b1 -> exact GELU -> dot with w2 over this tile's hidden units
     float part[8];
 #pragma unroll
@@ -246,6 +263,31 @@ __global__ void score_mlp_finish_kernel(const float* __restrict__ partial, int N
     probability_map(s, i, B, q_lut, score, prob, bin, q);
 }
 
+// One warp per rollout: u_j = b1_j + sum over the K splits, s = sum_j w2_j gelu(u_j) + b2 (lanes stride over j, fixed
+// shuffle order), then the probability map.
+template <typename T>
+__global__ void __launch_bounds__(128)
+score_mlp_splitk_finish_kernel(const float* __restrict__ upart, int splits, int N, int h, const T* __restrict__ b1,
+                               const T* __restrict__ w2, const T* __restrict__ b2, int B,
+                               const float* __restrict__ q_lut, float* score, float* prob, int32_t* bin, float* q) {
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (i >= N) return;
+    float s = 0.f;
+    for (int j = lane; j < h; j += 32) {
+        float u = b1 ? to_f32(b1[j]) : 0.f;
+        for (int z = 0; z < splits; ++z) u += upart[((int64_t)z * N + i) * h + j];
+        const float g = 0.5f * u * (1.0f + erff(u * 0.70710678118654752440f));
+        s = fmaf(to_f32(w2[j]), g, s);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+        if (b2) s += to_f32(b2[0]);
+        probability_map(s, i, B, q_lut, score, prob, bin, q);
+    }
+}
+
 template <typename T>
 int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index, int N,
                  const arrol_head* head, int B, const float* q_lut, float* score, float* prob, int32_t* bin,
@@ -260,14 +302,31 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
         ctx->launches += 1;
     } else {
         const int h_tiles = (head->h + TH - 1) / TH;
-        dim3 grid((N + TM - 1) / TM, h_tiles);
-        score_mlp_tile_kernel<T><<<grid, MLP_THREADS, 0, s>>>(hid, row_stride, row_index, N, head->d, head->h,
-                                                     static_cast<const T*>(head->W1),
-                                                     static_cast<const T*>(head->b1),
-                                                     static_cast<const T*>(head->w2), ctx->d_scratch, nullptr);
-        score_mlp_finish_kernel<T><<<(N + 255) / 256, 256, 0, s>>>(ctx->d_scratch, N, h_tiles,
-                                                                  static_cast<const T*>(head->b2), B, q_lut,
-                                                                  score, prob, bin, q);
+        const int m_tiles = (N + TM - 1) / TM;
+        // split d across blocks until there are about three blocks per SM, as far as the scratch allows
+        int splits = (3 * ctx->sm_count + m_tiles * h_tiles - 1) / (m_tiles * h_tiles);
+        if (splits > 8) splits = 8;
+        const size_t per_split = (size_t)N * (size_t)head->h;
+        while (splits > 1 && per_split * splits > ARROL_SCRATCH_FLOATS) --splits;
+        int k_len = ((head->d + splits - 1) / splits + TK - 1) / TK * TK;
+        splits = (head->d + k_len - 1) / k_len;
+        if (per_split * splits <= ARROL_SCRATCH_FLOATS) {
+            dim3 grid(m_tiles, h_tiles, splits);
+            score_mlp_tile_kernel<T, true><<<grid, MLP_THREADS, 0, s>>>(
+                hid, row_stride, row_index, N, head->d, head->h, static_cast<const T*>(head->W1), nullptr, nullptr,
+                ctx->d_scratch, nullptr, k_len);
+            score_mlp_splitk_finish_kernel<T><<<(N + 3) / 4, 128, 0, s>>>(
+                ctx->d_scratch, splits, N, head->h, static_cast<const T*>(head->b1), static_cast<const T*>(head->w2),
+                static_cast<const T*>(head->b2), B, q_lut, score, prob, bin, q);
+        } else {   // N x h too large for the scratch: one block per tile finishes its tile itself
+            dim3 grid(m_tiles, h_tiles);
+            score_mlp_tile_kernel<T, false><<<grid, MLP_THREADS, 0, s>>>(
+                hid, row_stride, row_index, N, head->d, head->h, static_cast<const T*>(head->W1),
+                static_cast<const T*>(head->b1), static_cast<const T*>(head->w2), ctx->d_scratch, nullptr, 0);
+            score_mlp_finish_kernel<T><<<(N + 255) / 256, 256, 0, s>>>(ctx->d_scratch, N, h_tiles,
+                                                                      static_cast<const T*>(head->b2), B, q_lut,
+                                                                      score, prob, bin, q);
+        }
         ctx->launches += 2;
     }
     ARROL_CUDA_OK(cudaGetLastError());
@@ -282,15 +341,15 @@ int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_str
     const int h_tiles = (head->h + TH - 1) / TH;
     dim3 grid((N + TM - 1) / TM, h_tiles);
     if (head->dtype == ARROL_F32)
-        score_mlp_tile_kernel<float><<<grid, MLP_THREADS, 0, s>>>(
+        score_mlp_tile_kernel<float, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const float*>(hidden), row_stride, row_index, N, head->d, head->h,
             static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
-            static_cast<const float*>(head->w2), partial, u_out);
+            static_cast<const float*>(head->w2), partial, u_out, 0);
     else
-        score_mlp_tile_kernel<__nv_bfloat16><<<grid, MLP_THREADS, 0, s>>>(
+        score_mlp_tile_kernel<__nv_bfloat16, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const __nv_bfloat16*>(hidden), row_stride, row_index, N, head->d, head->h,
             static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
-            static_cast<const __nv_bfloat16*>(head->w2), partial, u_out);
+            static_cast<const __nv_bfloat16*>(head->w2), partial, u_out, 0);
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
@@ -391,17 +450,17 @@ extern "C" int arrol_score_partial_static(const void* hidden, int64_t row_stride
     // The tile kernel writes every entry [tile][i], i < N, that the finishing kernel reads, so nothing left in
     // the array by an earlier call is ever read and nothing needs clearing.
     if (head->dtype == ARROL_F32) {
-        score_mlp_tile_kernel<float><<<grid, MLP_THREADS, 0, s>>>(
+        score_mlp_tile_kernel<float, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const float*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
-            static_cast<const float*>(head->w2), partial, nullptr);
+            static_cast<const float*>(head->w2), partial, nullptr, 0);
         score_mlp_finish_kernel<float><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const float*>(head->b2), B, q_lut, score, prob, bin, q);
     } else {
-        score_mlp_tile_kernel<__nv_bfloat16><<<grid, MLP_THREADS, 0, s>>>(
+        score_mlp_tile_kernel<__nv_bfloat16, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const __nv_bfloat16*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
-            static_cast<const __nv_bfloat16*>(head->w2), partial, nullptr);
+            static_cast<const __nv_bfloat16*>(head->w2), partial, nullptr, 0);
         score_mlp_finish_kernel<__nv_bfloat16><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const __nv_bfloat16*>(head->b2), B, q_lut, score, prob, bin, q);
     }
