@@ -150,6 +150,42 @@ int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab,
                         int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                         float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- Prune step in one call (Algorithm 1: quality check at the detection length, filter, re-batch) ----------
+ * arrol_score_partial -> arrol_select -> arrol_compact issued back to back on `stream` with N = P * G; every field
+ * has the meaning, layout and nullability of the argument of the same name in those calls.  Asynchronous. */
+typedef struct arrol_prune_step_args {
+    /* scoring */
+    const void* hidden;
+    int64_t row_stride_elems;
+    const int64_t* row_index;
+    arrol_head head;
+    arrol_calib calib;
+    float *score, *prob, *q;
+    int32_t* bin;
+    /* selection */
+    int32_t P, G, K, ddof;
+    double rho;
+    uint8_t* keep;
+    /* compaction */
+    const int32_t* lengths;
+    const int64_t* src_tok_off;
+    const int32_t* src_tokens;
+    const void* src_rows;
+    const float* rewards;
+    int64_t dst_capacity_tokens;
+    int32_t row_bytes;
+    float eps;
+    int32_t* dst_tokens;
+    void* dst_rows;
+    int64_t* cu_seqlens;
+    int32_t* survivor_idx;
+    float* adv;
+    float* tok_adv;
+    int32_t* tok_seq;
+    int64_t* d_num;
+} arrol_prune_step_args;
+int arrol_prune_step(arrol_ctx* ctx, const arrol_prune_step_args* args, void* stream);
+
 /* ---- Online calibrator and the deployed stochastic rule (Appendix A.4; Algorithm 1, backend) ----------
  * The calibrator state lives in ONE caller-provided device buffer of arrol_calib_state_bytes(B, cap) bytes
  * (16-byte aligned): two first-in-first-out rings of `cap` bin indices (positive / negative rollouts), their

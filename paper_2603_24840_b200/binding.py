@@ -26,6 +26,7 @@ EXPORTS = [
     "arrol_calib_delta", "arrol_select_stochastic",
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
     "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
+    "arrol_prune_step",
 ]
 
 
@@ -60,6 +61,17 @@ class _HostStep(C.Structure):
                 ("d_logp", C.c_void_p), ("d_workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("h_logp", C.c_void_p), ("h_adv", C.c_void_p), ("h_cu_seqlens", C.c_void_p),
                 ("h_survivor_idx", C.c_void_p), ("h_num", C.c_void_p)]
+
+
+class _PruneStep(C.Structure):
+    _fields_ = [("hidden", C.c_void_p), ("row_stride_elems", C.c_int64), ("row_index", C.c_void_p), ("head", _Head),
+                ("calib", _Calib), ("score", C.c_void_p), ("prob", C.c_void_p), ("q", C.c_void_p), ("bin", C.c_void_p),
+                ("P", C.c_int32), ("G", C.c_int32), ("K", C.c_int32), ("ddof", C.c_int32), ("rho", C.c_double),
+                ("keep", C.c_void_p), ("lengths", C.c_void_p), ("src_tok_off", C.c_void_p), ("src_tokens", C.c_void_p),
+                ("src_rows", C.c_void_p), ("rewards", C.c_void_p), ("dst_capacity_tokens", C.c_int64),
+                ("row_bytes", C.c_int32), ("eps", C.c_float), ("dst_tokens", C.c_void_p), ("dst_rows", C.c_void_p),
+                ("cu_seqlens", C.c_void_p), ("survivor_idx", C.c_void_p), ("adv", C.c_void_p), ("tok_adv", C.c_void_p),
+                ("tok_seq", C.c_void_p), ("d_num", C.c_void_p)]
 
 
 _lib = None
@@ -102,6 +114,8 @@ def load_library():
                                                C.POINTER(_Calib), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_void_p]
     lib.arrol_score_partial_static.restype = C.c_int
+    lib.arrol_prune_step.argtypes = [C.c_void_p, C.POINTER(_PruneStep), C.c_void_p]
+    lib.arrol_prune_step.restype = C.c_int
     lib.arrol_launch_count.argtypes = [C.c_void_p]
     lib.arrol_launch_count.restype = C.c_int64
     for fn in ("arrol_create", "arrol_destroy", "arrol_poll_status", "arrol_calib_counts", "arrol_build_q_lut",
@@ -308,3 +322,24 @@ def arrol_score_partial_static(hidden: torch.Tensor, head: dict, N: int, score: 
     _check(load_library().arrol_score_partial_static(_ptr(hidden), stride, _ptr(row_index), int(N), C.byref(hs),
                                                      C.byref(cs), _ptr(score), _ptr(prob), _ptr(bin), _ptr(q),
                                                      _stream(stream)), "arrol_score_partial_static")
+
+
+def make_prune_step(hidden: torch.Tensor, head: dict, q_lut: Optional[torch.Tensor], scalars: dict, tensors: dict,
+                    row_stride: Optional[int] = None) -> _PruneStep:
+    """Argument block of arrol_prune_step.  scalars: P, G, K, rho, eps, ddof, dst_capacity_tokens, row_bytes;
+    tensors: the device tensors by field name (missing / None = NULL).  The caller keeps the tensors alive."""
+    a = _PruneStep()
+    a.hidden = hidden.data_ptr()
+    a.row_stride_elems = hidden.stride(-2) if row_stride is None else int(row_stride)
+    _fill_head(a.head, _dtype_code(hidden), hidden.shape[-1], head)
+    a.calib.B = 0 if q_lut is None else q_lut.shape[0]
+    a.calib.q_lut = None if q_lut is None else q_lut.data_ptr()
+    for k, v in scalars.items():
+        setattr(a, k, v)
+    for k, t in tensors.items():
+        setattr(a, k, None if t is None else t.data_ptr())
+    return a
+
+
+def arrol_prune_step(ctx: Context, args: _PruneStep, stream=None):
+    _check(load_library().arrol_prune_step(ctx.handle, C.byref(args), _stream(stream)), "arrol_prune_step")

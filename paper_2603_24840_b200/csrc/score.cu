@@ -216,8 +216,7 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
             if (m < N && j < h)     // h % 4 == 0: a float4 never straddles the edge
                 *reinterpret_cast<float4*>(out + (int64_t)m * h + j) = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
         }
-        return;
-    }
+    } else {
     // epilogue: u + b1 -> exact GELU -> dot with w2 over this tile's hidden units
     float part[8];
 #pragma unroll
@@ -248,6 +247,7 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
             const int m = m0 + ty * 8 + a;
             if (m < N) partial[(int64_t)blockIdx.y * N + m] = part[a];
         }
+    }
     }
 }
 

@@ -106,6 +106,19 @@ class PruneRebatch:
         self.select()
         self.compact(with_rows)
 
+    def prune_step_args(self, with_rows: Optional[bool] = None):
+        """Argument block of the one-call prune step (arrol_prune_step) over this state's buffers."""
+        rows = self.with_rows if with_rows is None else with_rows
+        scal = dict(P=self.w.P, G=self.w.G, K=self.w.K, rho=self.w.rho, eps=1e-6, ddof=0,
+                    dst_capacity_tokens=self.cap, row_bytes=self.w.d * 2 if rows else 0)
+        tensors = dict(row_index=self.row_index, score=self.score, prob=self.prob, q=self.q, bin=self.bin,
+                       keep=self.keep, lengths=self.lengths, src_tok_off=self.src_tok_off,
+                       src_tokens=self.src_tokens, src_rows=self.src_rows if rows else None, rewards=self.rewards,
+                       dst_tokens=self.dst_tokens, dst_rows=self.dst_rows if rows else None,
+                       cu_seqlens=self.cu_seqlens, survivor_idx=self.survivor_idx, adv=self.adv,
+                       tok_adv=self.tok_adv, tok_seq=self.tok_seq, d_num=self.d_num)
+        return B.make_prune_step(self.hidden_score, self.head, self.q_lut, scal, tensors)
+
     def step(self):
         """One pass of the whole path: score -> select -> compact (tokens + hidden rows) -> token log-prob."""
         self.prune_step()
