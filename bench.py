@@ -27,10 +27,10 @@ sys.path.insert(0, ROOT)
 METRIC = "survivor_logprob_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM traffic of one token_logprob launch per survivor token at d = 2048, V = 128256 (two vocabulary splits), from
-# the ncu capture summarised in profiles/token_logprob_kernel_profile-small.md: (4.531 GB read + 7.5 MB written) /
+# DRAM traffic of one token_logprob launch per survivor token at d = 2048, V = 128256 (one vocabulary split), from
+# the ncu capture summarised in profiles/token_logprob_kernel_profile-small.md: (2.433 GB read + 5.4 MB written) /
 # 75,382 tokens.  At fixed d, V and split count the traffic grows in proportion to the tokens of the launch.
-LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256): 60200.0}
+LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256): 32340.0}
 
 
 def logprob_traffic(w, T, splits, sm_count):
@@ -331,8 +331,7 @@ def run_ours(args, w):
         achieved = flops / (logp_ms * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
         gather_bytes = 2.0 * T * w.d * 2 + 8.0 * T
-        ws_bytes = pr.workspace.numel()
-        splits = max(1, (ws_bytes - 256) // (16 * pr.cap)) if ws_bytes > 256 else 1
+        splits = B.arrol_token_logprob_splits(pr.ctx, pr.cap, w.d, w.V)
         traffic, traffic_src = logprob_traffic(w, T, splits, torch.cuda.get_device_properties(local).multi_processor_count)
         roofline = {
             "kernel": "token_logprob_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,

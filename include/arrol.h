@@ -144,8 +144,11 @@ int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths, c
  * logp float [T_max]; lse float [T_max] or NULL.  Both pointers 16-byte aligned; d % 8 == 0; inv_temperature > 0.
  * workspace: device scratch of at least arrol_token_logprob_workspace(ctx, T_max, d, V) bytes, 256-byte
  * aligned (holds per-split running maxima / sums when the vocabulary is split across thread blocks); its
- * contents need not be initialised and are undefined afterwards. */
+ * contents need not be initialised and are undefined afterwards.  The size is monotone in T_max: a workspace sized
+ * for T_max also serves calls on fewer tokens with the same d and V. */
 size_t arrol_token_logprob_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
+/* Number of vocabulary splits a launch on T_max tokens uses (1 = every block walks the whole vocabulary). */
+int32_t arrol_token_logprob_splits(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
 int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
                         int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                         float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);

@@ -26,7 +26,7 @@ EXPORTS = [
     "arrol_calib_delta", "arrol_select_stochastic",
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
     "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
-    "arrol_prune_step",
+    "arrol_prune_step", "arrol_token_logprob_splits",
 ]
 
 
@@ -255,6 +255,13 @@ def arrol_compact(ctx: Context, keep, lengths, src_tok_off, N: int, G: int, rewa
 
 def arrol_token_logprob_workspace(ctx: Context, T_max: int, d: int, V: int) -> int:
     return int(load_library().arrol_token_logprob_workspace(ctx.handle, int(T_max), int(d), int(V)))
+
+
+def arrol_token_logprob_splits(ctx: Context, T_max: int, d: int, V: int) -> int:
+    lib = load_library()
+    lib.arrol_token_logprob_splits.restype = C.c_int32
+    lib.arrol_token_logprob_splits.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32]
+    return int(lib.arrol_token_logprob_splits(ctx.handle, int(T_max), int(d), int(V)))
 
 
 def arrol_token_logprob(ctx: Context, hidden, W_vocab, targets, T_max: int, d: int, V: int, logp, workspace,
