@@ -25,8 +25,9 @@ constexpr int B_STAGE_BYTES = BN * BK * 2;
 constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int MN_BLOCK_BYTES = BK * 128;   // one 64-element MN block of an MN-major stage: BK rows of 128 bytes
 constexpr int TMEM_COLS = 512;
-constexpr int NUM_THREADS = 192;
-constexpr int EPI_WARPS = 4;
+constexpr int EPI_WARPS = 8;            // two warps per tensor-memory lane quarter, each takes half of the columns
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
+constexpr int EPI_PIECES = BN / 32 / (EPI_WARPS / 4);   // 32-column pieces per epilogue warp and accumulator
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
 constexpr int TC = 74 * BM;      // tokens per chunk: 74 token tiles, so that TC/128 x d/256 tiles fill 148 SMs evenly
 
@@ -254,6 +255,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
         }
     } else {
         const int quarter = warp & 3;
+        const int col_half = (warp - 2) >> 2;           // 0 or 1: which half of the accumulator's columns
         const int row_in_tile = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint32_t acc = 0, acc_phase = 0;
@@ -315,14 +317,15 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                     }
                 };
                 uint32_t ra[32], rb[32];
-                tcgen05_ld_32x32_issue(tacc, ra);
+                const int p0 = col_half * EPI_PIECES, p1 = p0 + EPI_PIECES;   // this warp's pieces of the accumulator
+                tcgen05_ld_32x32_issue(tacc + p0 * 32, ra);
 #pragma unroll 1
-                for (int piece = 0; piece < BN / 32; piece += 2) {
+                for (int piece = p0; piece < p1; piece += 2) {
                     tcgen05_ld_wait(ra);
                     tcgen05_ld_32x32_issue(tacc + (piece + 1) * 32, rb);
                     emit(ra, piece);
                     tcgen05_ld_wait(rb);
-                    if (piece + 2 < BN / 32) tcgen05_ld_32x32_issue(tacc + (piece + 2) * 32, ra);
+                    if (piece + 2 < p1) tcgen05_ld_32x32_issue(tacc + (piece + 2) * 32, ra);
                     emit(rb, piece + 1);
                 }
                 tcgen05_fence_before();
@@ -380,6 +383,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         }
     } else {
         const int quarter = warp & 3;
+        const int col_half = (warp - 2) >> 2;           // 0 or 1: which half of the accumulator's columns
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
@@ -392,7 +396,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             tcgen05_fence_after();
             float* crow = p.C + (int64_t)row * p.ldc;
 #pragma unroll 1
-            for (int piece = 0; piece < BN / 32; ++piece) {
+            for (int piece = col_half * EPI_PIECES; piece < (col_half + 1) * EPI_PIECES; ++piece) {
                 const int pc0 = col0 + piece * 32;
                 if (pc0 >= p.N) break;
                 float v[32];
