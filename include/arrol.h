@@ -242,10 +242,10 @@ int arrol_select_stochastic(arrol_ctx* ctx, const float* q, const float* u, cons
  *     cores;  dH [T_max, d] float = dz W_vocab (rows t >= T are zero or left untouched);  dW [V, d] float = dz^T hidden
  *     (overwritten).  Positions with targets[t] < 0 or >= V carry no gradient.  dz is rounded to bf16 before the two
  *     contractions.  hidden, W_vocab, targets, T_max, d_T, d, V as in arrol_token_logprob; dH, dW 16-byte aligned.
- *   hidden rows t in [T, T_max) are multiplied by zero gradients where the last live 64-row block is contracted:
- *   they must hold finite values (any finite bit pattern, e.g. zeros or stale rows).
+ *   hidden rows t in [T, T_max) are never read by the contractions (the last, partly live block of rows goes
+ *   through a zero-padded copy), so they may hold anything.
  *   workspace: arrol_lm_head_backward_workspace(ctx, T_max, d, V) bytes, 256-byte aligned (one chunk of 9,472 tokens
- *   of dz in bf16): 9472 * 2 * V bytes (V rounded up to 8). */
+ *   of dz in bf16 and one 64-row block of hidden): 9472 * 2 * V + 128 * d bytes (V rounded up to 8). */
 int arrol_policy_loss(arrol_ctx* ctx, const float* logp, const float* logp_old, const float* logp_ref,
                       const float* tok_adv, const int32_t* tok_seq, const int64_t* cu_seqlens, const int64_t* d_num,
                       int64_t T_max, float eps_low, float eps_high, float beta, int32_t agg_mode, float* grad_logp,

@@ -93,7 +93,8 @@ __device__ __forceinline__ void pipe_teardown(const PipeSmem& ps, uint32_t tmem_
 //   MN-major operand: MN/64 boxes [64 K rows x 64 MN columns]     at (x = mn0 + 64 b, y = k), BK*128 bytes apart.
 template <bool A_MN, bool B_MN, int PF, typename Coords>
 __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensorMap* ma, const CUtensorMap* mb,
-                                              int k_steps, Coords coords) {
+                                              int k_steps, Coords coords, const CUtensorMap* mb_tail = nullptr,
+                                              int tail_ks = -1) {
     uint32_t stage = 0, phase = 0, issued = 0;
     bool ok = true;
     int ay, by;
@@ -128,7 +129,11 @@ __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensor
             }
             if constexpr (B_MN) {
 #pragma unroll
-                for (int b = 0; b < BN / 64; ++b) tma_load_2d(sb + b * MN_BLOCK_BYTES, mb, by + 64 * b, ks * BK, &ps.full[stage]);
+                for (int b = 0; b < BN / 64; ++b) {
+                    // the K step that holds the last, partly live block of rows is read from its zero-padded copy
+                    if (ks == tail_ks) tma_load_2d(sb + b * MN_BLOCK_BYTES, mb_tail, by + 64 * b, 0, &ps.full[stage]);
+                    else tma_load_2d(sb + b * MN_BLOCK_BYTES, mb, by + 64 * b, ks * BK, &ps.full[stage]);
+                }
             } else {
                 tma_load_2d(sb, mb, ks * BK, by, &ps.full[stage]);
             }
@@ -354,7 +359,8 @@ struct GemmParams {
 
 template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const GemmParams p) {
+gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+            const __grid_constant__ CUtensorMap map_b_tail, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const PipeSmem ps = carve_smem(smem_raw);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -368,13 +374,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
 
     if (warp == 0) {
         if (lane == 0) {
+            const int tail_ks = (p.k_is_tokens && (K % BK) != 0) ? k_steps - 1 : -1;
             producer_loop<A_MN, B_MN, 0>(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
                 const int64_t item = blockIdx.x + it * gridDim.x;
                 if (item >= items) return false;
                 ay = (int)(item / n_tiles) * BM;       // consecutive blocks share the A panel, walk the B panels
                 by = (int)(item % n_tiles) * BN;
                 return true;
-            });
+            }, &map_b_tail, tail_ks);
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -429,16 +436,31 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     pipe_teardown(ps, tmem_base, p.d_status);
 }
 
+// Copies the last, partly live 64-row block of the chunk's hidden rows into `tail` [64, d] and pads it with zeros,
+// so that rows past the live tokens (caller memory that may hold anything) never reach the tensor core.
+__global__ void tail_block_kernel(const uint16_t* __restrict__ hidden, int d, const int64_t* d_T, int64_t T_max,
+                                  int64_t t0, uint16_t* __restrict__ tail) {
+    const int64_t T = live_tokens(d_T, T_max);
+    if (t0 >= T) return;
+    const int64_t live = min((int64_t)TC, T - t0);
+    const int64_t r0 = live / BK * BK;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < (int64_t)BK * d; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / d, c = i - r * d;
+        tail[i] = (r0 + r < live) ? hidden[(t0 + r0 + r) * d + c] : (uint16_t)0;
+    }
+}
+
 struct BackwardLayout {
     int64_t ldz;       // V rounded up to 8
-    size_t dz, total;
+    size_t dz, tail, total;
 };
 
-BackwardLayout backward_layout(int V) {
+BackwardLayout backward_layout(int d, int V) {
     BackwardLayout L;
     L.ldz = ((int64_t)V + 7) & ~(int64_t)7;
     L.dz = 0;
-    L.total = (((size_t)TC * L.ldz * 2) + 255) & ~(size_t)255;
+    L.tail = (((size_t)TC * L.ldz * 2) + 255) & ~(size_t)255;
+    L.total = L.tail + (((size_t)BK * d * 2 + 255) & ~(size_t)255);
     return L;
 }
 
@@ -446,7 +468,7 @@ BackwardLayout backward_layout(int V) {
 
 extern "C" size_t arrol_lm_head_backward_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
     if (!ctx || T_max <= 0 || d <= 0 || V <= 0) return 0;
-    return backward_layout(V).total;
+    return backward_layout(d, V).total;
 }
 
 extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
@@ -465,9 +487,10 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     if (!hidden || !W_vocab || !targets || !grad_logp || !lse || !dH) return ARROL_ERR_INVALID_ARG;
     if (!arrol_aligned(hidden, 16) || !arrol_aligned(W_vocab, 16) || !arrol_aligned(dH, 16) || !arrol_aligned(dW, 16))
         return ARROL_ERR_INVALID_ARG;
-    const BackwardLayout L = backward_layout(V);
+    const BackwardLayout L = backward_layout(d, V);
     if (!workspace || workspace_bytes < L.total || !arrol_aligned(workspace, 256)) return ARROL_ERR_WORKSPACE;
     __nv_bfloat16* dZ = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + L.dz);
+    uint16_t* Htail = reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + L.tail);
 
     ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
@@ -475,12 +498,14 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
 
     // tensor maps: K-major operands are fetched as [MN rows x 64 K columns] boxes, MN-major ones as [64 K rows x 64 MN
     // columns] boxes of the same row-major storage
-    CUtensorMap map_h_k, map_w_k, map_dz_k, map_w_mn, map_dz_mn, map_h_mn;
+    CUtensorMap map_h_k, map_w_k, map_dz_k, map_w_mn, map_dz_mn, map_h_mn, map_h_tail;
     if (make_map(ctx, &map_h_k, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map(ctx, &map_w_k, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map_ld(ctx, &map_dz_k, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map_ld(ctx, &map_dz_mn, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+
+    if (make_map(ctx, &map_h_tail, Htail, (uint64_t)BK, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
 
     const int total_chunks = (V + BN - 1) / BN;
     int splits = 1;
@@ -509,14 +534,15 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
         gh.d_T = d_T; gh.T_max = T_max; gh.t0 = t0; gh.d_status = ctx->d_status;
         const int64_t gh_items = (int64_t)((rows + BM - 1) / BM) * ((d + BN - 1) / BN);
         gemm_kernel<false, true><<<(unsigned)(gh_items < ctx->sm_count ? gh_items : ctx->sm_count), NUM_THREADS,
-                                   SMEM_BYTES, s>>>(map_dz_k, map_w_mn, gh);
+                                   SMEM_BYTES, s>>>(map_dz_k, map_w_mn, map_w_mn, gh);
+        tail_block_kernel<<<64, 256, 0, s>>>(static_cast<const uint16_t*>(hidden), d, d_T, T_max, t0, Htail);
         GemmParams gw;    // dW += dZ^T . H[chunk]
         gw.M = V; gw.N = d; gw.K = (int)rows; gw.C = dW; gw.ldc = d; gw.accumulate = 1; gw.k_is_tokens = 1;
         gw.d_T = d_T; gw.T_max = T_max; gw.t0 = t0; gw.d_status = ctx->d_status;
         const int64_t gw_items = (int64_t)((V + BM - 1) / BM) * ((d + BN - 1) / BN);
         gemm_kernel<true, true><<<(unsigned)(gw_items < ctx->sm_count ? gw_items : ctx->sm_count), NUM_THREADS,
-                                  SMEM_BYTES, s>>>(map_dz_mn, map_h_mn, gw);
-        ctx->launches += 3;
+                                  SMEM_BYTES, s>>>(map_dz_mn, map_h_mn, map_h_tail, gw);
+        ctx->launches += 4;
         ARROL_CUDA_OK(cudaGetLastError());
     }
     return ARROL_OK;

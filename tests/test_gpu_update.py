@@ -66,6 +66,8 @@ def _backward_case(ctx, T, d, V, seed, T_live=None, inv_temp=1.0):
     dH_ref, dW_ref = ou.lm_head_backward(synth.as_oracle_array(H[:n]), synth.as_oracle_array(W), y[:n],
                                          gl[:n].astype(np.float64), inv_temp=inv_temp)
     Hd, Wd, yd = H.cuda(), W.cuda(), dv(y)
+    if T_live is not None:
+        Hd[T_live:] = float("nan")               # rows past the live tokens may hold anything
     logp = torch.empty(T, device="cuda")
     lse = torch.empty(T, device="cuda")
     d_T = None if T_live is None else torch.tensor([T_live], dtype=torch.int64, device="cuda")
@@ -96,6 +98,8 @@ def test_lm_head_backward_many_chunks_temperature_and_device_T(ctx):
     _backward_case(ctx, 400, 128, 1024, seed=2, inv_temp=0.6)
     dH, n = _backward_case(ctx, 600, 128, 1024, seed=3, T_live=333)
     assert np.all(dH[n:] == 0.0)                               # rows past T inside a processed chunk are zero
+    _backward_case(ctx, 600, 128, 1024, seed=4, T_live=320)    # live rows end exactly on a 64-row block
+    _backward_case(ctx, 9700, 64, 512, seed=5, T_live=9500)    # the partly live block is in the second chunk
 
 
 def test_update_argument_errors(ctx):
