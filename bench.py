@@ -283,7 +283,7 @@ def run_ours(args, w):
         prune_us[label] = a.elapsed_time(b) / reps * 1e3
 
     # scoring kernel on its own: the linear head streamed over every source row (HBM-bound: d*e bytes per row);
-    # the MLP head on the workload's own N rollouts (fp32-ALU-bound: 2*d*h flops per row)
+    # the MLP head on the workload's own N rollouts (2*d*h flops per row, on the tensor cores for bf16 heads)
     n_score = min(pr.T_src, 1 << 20) if w.h == 0 else w_rank.N
     so = [torch.empty(n_score, dtype=torch.float32, device=pr.dev) for _ in range(3)]
     ridx = None if w.h == 0 else pr.row_index
@@ -380,11 +380,14 @@ def run_ours(args, w):
                                              "scores only N = %d rows (launch-latency bound)" % w_rank.N}
         else:
             tfs = 2.0 * n_score * w.d * w.h / (score_ms * 1e-3) / 1e12
-            alu_peak = 2.0 * 128 * props.multi_processor_count * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
-            out["score_roofline"] = {"kernel": "score_mlp_tile_kernel", "bound": "alu", "rows": int(n_score),
-                                     "achieved": tfs, "peak": alu_peak, "unit": "TFLOP/s", "frac": tfs / alu_peak,
-                                     "launch_ms": score_ms,
-                                     "note": "fp32 FMA roof = 2 x 128 lanes x SMs x max SM clock"}
+            tc_peak = float(peaks["bf16_tflops"])
+            out["score_roofline"] = {"kernel": "pack_rows_kernel + score_mlp_tc_kernel", "bound": "tensor",
+                                     "rows": int(n_score), "achieved": tfs, "peak": tc_peak, "unit": "TFLOP/s",
+                                     "frac": tfs / tc_peak, "launch_ms": score_ms,
+                                     "note": "2*N*d*h flops of the head's first layer over the whole call (row packing, "
+                                             "contraction, GELU, probability map); a few GFLOP on %d blocks: bound by "
+                                             "launch and pipeline latency, not by the tensor pipe"
+                                             % (((n_score + 127) // 128) * ((w.h + 63) // 64))}
         if update is not None:
             upd_flops = 6.0 * T * w.d * w.V
             out["update"] = {"what": "arrol_policy_loss + arrol_lm_head_backward on the step's survivors "

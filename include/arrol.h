@@ -55,8 +55,10 @@ int arrol_version(void);                    /* major*10000 + minor*100 + patch *
 const char* arrol_status_string(int status); /* static string, never NULL */
 
 /* Creates a context on CUDA device `device` (made current for the calling thread during the call).
- * Allocates the context's device status word, a 16 MB scratch buffer, 1 MB of pinned host memory, a second
- * stream and a few events (used by arrol_prune_rebatch_host); nothing is allocated later. */
+ * Allocates the context's device status word, a 16 MB scratch buffer and a 64 MB row-packing buffer (MLP head),
+ * 1 MB of pinned host memory, a second stream and a few events (used by arrol_prune_rebatch_host); nothing is
+ * allocated later.  Calls that use the context's buffers (MLP-head scoring, the policy loss, the head training
+ * step) must be ordered on the device with respect to one another, e.g. by issuing them on one stream. */
 int arrol_create(arrol_ctx** out, int device);
 int arrol_destroy(arrol_ctx* ctx);
 
@@ -96,6 +98,8 @@ typedef struct arrol_calib {
  *   score[i] = head(x);  prob[i] = s' = 1 / (1 + exp(-score[i]));
  *   bin[i] = min(B-1, floor(B s'));  q[i] = q_lut[bin[i]]   (q[i] = s' when there is no table).
  * Outputs: score, prob, q float [N] (required); bin int32 [N] or NULL.  fp32 accumulation.
+ * A bf16 MLP head runs its first layer on the tensor cores (bf16 products, fp32 accumulation); rows picked by
+ * row_index are first packed into the context's buffer.
  * row_index holds int64 row numbers; it must stay valid until the work completes.
  * Errors: INVALID_ARG for NULL/negative/misaligned arguments, UNSUPPORTED for d % 8 != 0, h % 4 != 0,
  * h > 4096, or N larger than the context scratch allows for the MLP head (65536). N == 0 is a no-op. */

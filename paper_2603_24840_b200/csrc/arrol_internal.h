@@ -14,6 +14,8 @@ struct arrol_ctx {
     uint32_t* d_status;        // device status word (bits ARROL_DEV_*)
     uint32_t* h_status;        // pinned host mirror used by arrol_poll_status
     float* d_scratch;          // MLP-head partial sums: [ARROL_SCRATCH_FLOATS]
+    void* d_pack;              // MLP head on the tensor cores: the scored rows packed as bf16 [N][d], ARROL_PACK_BYTES
+    uint32_t* d_tile_counters; // MLP head on the tensor cores: finished blocks per row tile, zero between calls
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
     unsigned long long launches;   // kernels launched through this context (host-side count)
     cudaStream_t copy_stream;      // second stream of the host-buffer step: uploads overlap the log-prob kernel
@@ -25,6 +27,8 @@ constexpr int ARROL_MAX_MLP_N = 65536;       // rollouts per arrol_score_partial
 constexpr int ARROL_MLP_TH = 64;             // hidden units per MLP thread-block tile
 constexpr int ARROL_MAX_H = 4096;
 constexpr size_t ARROL_SCRATCH_FLOATS = (size_t)ARROL_MAX_MLP_N * (ARROL_MAX_H / ARROL_MLP_TH);
+constexpr size_t ARROL_PACK_BYTES = (size_t)64 << 20;
+constexpr int ARROL_TILE_COUNTERS = 1024;
 
 #define ARROL_CUDA_OK(expr)                      \
     do {                                         \
@@ -55,3 +59,9 @@ struct ArrolDeviceGuard {
 // score.cu: MLP tile pass with optional pre-activation output; partial is [ceil(h / ARROL_MLP_TH)][N].
 int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index, int N,
                              const arrol_head* head, float* partial, float* u_out, cudaStream_t s);
+
+// score_tc.cu: scores of a bf16 MLP head on the tensor cores (pack, contraction, GELU, w2 dot, probability map).
+// ARROL_ERR_UNSUPPORTED (nothing launched) when the sizes do not fit the context's buffers.
+int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index,
+                                int N, const arrol_head* head, int B, const float* q_lut, float* score, float* prob,
+                                int32_t* bin, float* q, cudaStream_t s);

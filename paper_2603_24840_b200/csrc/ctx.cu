@@ -42,6 +42,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->d_status = nullptr;
     ctx->h_status = nullptr;
     ctx->d_scratch = nullptr;
+    ctx->d_pack = nullptr;
+    ctx->d_tile_counters = nullptr;
     ctx->encode_tiled = nullptr;
     ctx->launches = 0;
     ctx->copy_stream = nullptr;
@@ -51,6 +53,9 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
               cudaMemset(ctx->d_status, 0, 256) == cudaSuccess &&
               cudaMallocHost(&ctx->h_status, 64) == cudaSuccess &&
               cudaMalloc(&ctx->d_scratch, ARROL_SCRATCH_FLOATS * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&ctx->d_pack, ARROL_PACK_BYTES) == cudaSuccess &&
+              cudaMalloc(&ctx->d_tile_counters, ARROL_TILE_COUNTERS * sizeof(uint32_t)) == cudaSuccess &&
+              cudaMemset(ctx->d_tile_counters, 0, ARROL_TILE_COUNTERS * sizeof(uint32_t)) == cudaSuccess &&
               cudaMallocHost(&ctx->h_keep, ARROL_MAX_HOST_N) == cudaSuccess &&
               cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; ok && i < ARROL_COPY_EVENTS; ++i)
@@ -77,6 +82,8 @@ extern "C" int arrol_destroy(arrol_ctx* ctx) {
     if (ctx->d_status) (void)cudaFree(ctx->d_status);
     if (ctx->h_status) (void)cudaFreeHost(ctx->h_status);
     if (ctx->d_scratch) (void)cudaFree(ctx->d_scratch);
+    if (ctx->d_pack) (void)cudaFree(ctx->d_pack);
+    if (ctx->d_tile_counters) (void)cudaFree(ctx->d_tile_counters);
     if (ctx->h_keep) (void)cudaFreeHost(ctx->h_keep);
     for (int i = 0; i < ARROL_COPY_EVENTS; ++i)
         if (ctx->copy_events[i]) (void)cudaEventDestroy(ctx->copy_events[i]);

@@ -11,6 +11,7 @@
 #include <cuda_bf16.h>
 
 #include "arrol_internal.h"
+#include "score_common.cuh"
 
 namespace {
 
@@ -54,21 +55,6 @@ template <> struct Vec16<__nv_bfloat16> {
         }
     }
 };
-
-// s -> s' = sigmoid(s), b = min(B-1, floor(B s')), q = q_lut[b] (Appendix A.4)
-__device__ __forceinline__ void probability_map(float s, int i, int B, const float* __restrict__ q_lut,
-                                                float* score, float* prob, int32_t* bin, float* q) {
-    float sp = 1.0f / (1.0f + expf(-s));
-    int b = 0;
-    if (B > 0) {
-        b = (int)floorf((float)B * sp);
-        b = min(max(b, 0), B - 1);
-    }
-    score[i] = s;
-    prob[i] = sp;
-    if (bin) bin[i] = b;
-    q[i] = (q_lut != nullptr) ? __ldg(q_lut + b) : sp;
-}
 
 template <typename T>
 __global__ void __launch_bounds__(128)
@@ -301,6 +287,13 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
             static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q);
         ctx->launches += 1;
     } else {
+        if constexpr (sizeof(T) == 2) {
+            // bf16 head: the first layer is a dense contraction, so the whole head runs on the tensor-core path
+            // when the context's buffers hold the problem
+            const int rc = arrol_internal_score_mlp_tc(ctx, hidden, row_stride, row_index, N, head, B, q_lut, score,
+                                                       prob, bin, q, s);
+            if (rc != ARROL_ERR_UNSUPPORTED) return rc;
+        }
         const int h_tiles = (head->h + TH - 1) / TH;
         const int m_tiles = (N + TM - 1) / TM;
         // split d across blocks until there are about three blocks per SM, as far as the scratch allows

@@ -94,10 +94,31 @@ def test_linear_head(ctx, N, d, dtype, use_lut, use_index):
     (300, 2048, 256, torch.bfloat16),
     (70, 264, 132, torch.float32),
     (129, 512, 512, torch.bfloat16),
+    (1000, 1024, 128, torch.bfloat16),      # several 128-row tiles and K ranges on the tensor-core path
+    (257, 200, 68, torch.bfloat16),         # d and h off the 64-wide tile edges
+    (2048, 2048, 256, torch.bfloat16),      # the Qwen-3-1.7B-shaped head
 ])
 def test_mlp_head(ctx, N, d, h, dtype):
     _score_case(ctx, N, d, h, dtype, True, True, seed=N + h)
     _score_case(ctx, N, d, h, dtype, False, False, seed=N + h + 1, bias=False)
+
+
+def test_mlp_head_strided_rows_without_index(ctx):
+    """Evenly strided rows (a column slice of a wider buffer) go to the tensor-core path without packing."""
+    g = np.random.default_rng(5)
+    N, d, h = 200, 256, 64
+    wide = torch.from_numpy(g.normal(size=(N, 2 * d)).astype(np.float32)).to(torch.bfloat16)
+    x = wide[:, :d]
+    mk = lambda *s: torch.from_numpy(g.normal(0, 0.05, size=s).astype(np.float32)).to(torch.bfloat16)
+    head = {"W1": mk(h, d), "b1": mk(h), "w2": mk(h) * 4, "b2": mk(1)}
+    oa = synth.as_oracle_array
+    s_ref = oracle.head_score(oa(x.contiguous()), oa(head["W1"]), oa(head["b1"]), oa(head["w2"]), oa(head["b2"]), h=h)
+    dhead = {k: v.cuda() for k, v in head.items()}
+    dhead["h"] = h
+    out = [torch.full((N,), 7.0, device="cuda") for _ in range(3)]
+    B.arrol_score_partial(ctx, wide.cuda()[:, :d], dhead, N, out[0], out[1], out[2])
+    torch.cuda.synchronize()
+    assert np.abs(out[0].cpu().numpy() - s_ref).max() <= PROB_TOL
 
 
 def test_score_argument_errors(ctx):
