@@ -90,49 +90,46 @@ __device__ __forceinline__ void pipe_teardown(const PipeSmem& ps, uint32_t tmem_
 // Producer role (one thread).  For every accumulator tile `coords(it, a_mn0, b_mn0)` gives the operands' MN
 // origins (it returns false when the tile list is exhausted); for every K step the stage receives
 //   K-major operand:  one box  [MN rows x 64 K columns]           at (x = k, y = mn0)
-//   MN-major operand: MN/64 boxes [64 K rows x 64 MN columns]     at (x = mn0 + 64 b, y = k), BK*128 bytes apart.
-template <bool A_MN, bool B_MN, int PF, typename Coords>
+//   MN-major operand: MN/64 blocks [64 K rows x 64 MN columns], BK*128 bytes apart: one three-dimensional box
+//                     (64 elements, 64 K rows, MN/64 blocks) at (0, k, mn0/64) when the map is of that kind
+//                     (a3d / b3d), else one two-dimensional box per block at (x = mn0 + 64 b, y = k).
+// Issuing a copy costs the thread about 60 cycles, and a stage's MMAs last 512: with one copy per operand the
+// producer keeps ahead of the tensor pipe, with six it does not.
+template <bool A_MN, bool B_MN, typename Coords>
 __device__ __forceinline__ void producer_loop(const PipeSmem& ps, const CUtensorMap* ma, const CUtensorMap* mb,
-                                              int k_steps, Coords coords, const CUtensorMap* mb_tail = nullptr,
-                                              int tail_ks = -1) {
+                                              int k_steps, Coords coords, bool a3d = false, bool b3d = false,
+                                              const CUtensorMap* mb_tail = nullptr, int tail_ks = -1) {
     uint32_t stage = 0, phase = 0, issued = 0;
     bool ok = true;
     int ay, by;
     for (int64_t it = 0; ok && coords(it, ay, by); ++it) {
         for (int ks = 0; ks < k_steps; ++ks) {
             if (!mbar_wait(&ps.empty[stage], phase ^ 1u, ps.abort_flag)) { ok = false; break; }
-            if constexpr (PF > 0) {   // pull the tiles PF steps ahead into L2 (operands that stream from HBM)
-                const int kp = (ks + PF) * BK;
-                if (ks + PF < k_steps) {
-                    if constexpr (A_MN) {
-#pragma unroll
-                        for (int b = 0; b < BM / 64; ++b) tma_prefetch_l2_2d(ma, ay + 64 * b, kp);
-                    } else {
-                        tma_prefetch_l2_2d(ma, kp, ay);
-                    }
-                    if constexpr (B_MN) {
-#pragma unroll
-                        for (int b = 0; b < BN / 64; ++b) tma_prefetch_l2_2d(mb, by + 64 * b, kp);
-                    } else {
-                        tma_prefetch_l2_2d(mb, kp, by);
-                    }
-                }
-            }
             mbar_expect_tx(&ps.full[stage], STAGE_BYTES);
             uint8_t* sa = ps.stage_a + (size_t)stage * A_STAGE_BYTES;
             uint8_t* sb = ps.stage_b + (size_t)stage * B_STAGE_BYTES;
             if constexpr (A_MN) {
+                if (a3d) {
+                    tma_load_3d(sa, ma, 0, ks * BK, ay >> 6, &ps.full[stage]);
+                } else {
 #pragma unroll
-                for (int b = 0; b < BM / 64; ++b) tma_load_2d(sa + b * MN_BLOCK_BYTES, ma, ay + 64 * b, ks * BK, &ps.full[stage]);
+                    for (int b = 0; b < BM / 64; ++b)
+                        tma_load_2d(sa + b * MN_BLOCK_BYTES, ma, ay + 64 * b, ks * BK, &ps.full[stage]);
+                }
             } else {
                 tma_load_2d(sa, ma, ks * BK, ay, &ps.full[stage]);
             }
             if constexpr (B_MN) {
+                // the K step that holds the last, partly live block of rows is read from its zero-padded copy
+                const bool tail = ks == tail_ks;
+                const CUtensorMap* m = tail ? mb_tail : mb;
+                const int ky = tail ? 0 : ks * BK;
+                if (b3d) {
+                    tma_load_3d(sb, m, 0, ky, by >> 6, &ps.full[stage]);
+                } else {
 #pragma unroll
-                for (int b = 0; b < BN / 64; ++b) {
-                    // the K step that holds the last, partly live block of rows is read from its zero-padded copy
-                    if (ks == tail_ks) tma_load_2d(sb + b * MN_BLOCK_BYTES, mb_tail, by + 64 * b, 0, &ps.full[stage]);
-                    else tma_load_2d(sb + b * MN_BLOCK_BYTES, mb, by + 64 * b, ks * BK, &ps.full[stage]);
+                    for (int b = 0; b < BN / 64; ++b)
+                        tma_load_2d(sb + b * MN_BLOCK_BYTES, m, by + 64 * b, ky, &ps.full[stage]);
                 }
             } else {
                 tma_load_2d(sb, mb, ks * BK, by, &ps.full[stage]);
@@ -235,7 +232,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
             int64_t item = blockIdx.x;
             int m_tile = 0, c = 0, c1 = 0;
             bool have = false;
-            producer_loop<false, false, 0>(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
+            producer_loop<false, false>(ps, &map_h, &map_w, k_steps, [&](int64_t, int& ay, int& by) {
                 while (!have || c >= c1) {
                     if (have) item += gridDim.x;
                     if (item >= items) return false;
@@ -352,6 +349,7 @@ struct GemmParams {
     int64_t ldc;
     int accumulate;           // 1: C += ..., 0: C = ...
     int k_is_tokens;          // 1: K counts the chunk's tokens: only the live ones (T - t0) are contracted
+    int a3d, b3d;             // the MN-major operand's maps are three-dimensional (one copy per stage)
     const int64_t* d_T;       // the launch is skipped when t0 >= live tokens
     int64_t T_max, t0;
     uint32_t* d_status;
@@ -375,13 +373,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
     if (warp == 0) {
         if (lane == 0) {
             const int tail_ks = (p.k_is_tokens && (K % BK) != 0) ? k_steps - 1 : -1;
-            producer_loop<A_MN, B_MN, 0>(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
+            producer_loop<A_MN, B_MN>(ps, &map_a, &map_b, k_steps, [&](int64_t it, int& ay, int& by) {
                 const int64_t item = blockIdx.x + it * gridDim.x;
                 if (item >= items) return false;
                 ay = (int)(item / n_tiles) * BM;       // consecutive blocks share the A panel, walk the B panels
                 by = (int)(item % n_tiles) * BN;
                 return true;
-            }, &map_b_tail, tail_ks);
+            }, p.a3d != 0, p.b3d != 0, &map_b_tail, tail_ks);
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -496,16 +494,23 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
 
-    // tensor maps: K-major operands are fetched as [MN rows x 64 K columns] boxes, MN-major ones as [64 K rows x 64 MN
-    // columns] boxes of the same row-major storage
+    // tensor maps: K-major operands are fetched as [MN rows x 64 K columns] boxes; MN-major ones (the same row-major
+    // storage read the other way) as one three-dimensional box per stage when the MN extent is a whole number of
+    // 64-element blocks, else as one [64 K rows x 64 MN columns] box per block
     CUtensorMap map_h_k, map_w_k, map_dz_k, map_w_mn, map_dz_mn, map_h_mn, map_h_tail;
     if (make_map(ctx, &map_h_k, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map(ctx, &map_w_k, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map_ld(ctx, &map_dz_k, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
-    if (make_map_ld(ctx, &map_dz_mn, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BK) != ARROL_OK) return ARROL_ERR_CUDA;
-
-    if (make_map(ctx, &map_h_tail, Htail, (uint64_t)BK, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+    bool d3 = d % 64 == 0, v3 = V % 64 == 0;
+    if (d3 && (make_map_mn3d(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN / 64) != ARROL_OK ||
+               make_map_mn3d(ctx, &map_h_tail, Htail, (uint64_t)BK, (uint64_t)d, (uint64_t)d, BN / 64) != ARROL_OK))
+        d3 = false;
+    if (v3 && make_map_mn3d(ctx, &map_dz_mn, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM / 64) != ARROL_OK) v3 = false;
+    if (!d3) {
+        if (make_map(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+        if (make_map(ctx, &map_h_tail, Htail, (uint64_t)BK, (uint64_t)d, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+    }
+    if (!v3 && make_map_ld(ctx, &map_dz_mn, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BK) != ARROL_OK) return ARROL_ERR_CUDA;
 
     const int total_chunks = (V + BN - 1) / BN;
     int splits = 1;
@@ -516,8 +521,9 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     for (int64_t t0 = 0; t0 < T_max; t0 += TC) {
         const int64_t rows = (T_max - t0) < TC ? (T_max - t0) : (int64_t)TC;
         // the chunk of hidden as an MN-major B operand: [rows (K), d (N)]; rows past T_max read as zero
-        if (make_map(ctx, &map_h_mn, static_cast<const uint8_t*>(hidden) + (size_t)t0 * d * 2, (uint64_t)rows, (uint64_t)d,
-                     BK) != ARROL_OK)
+        const void* h_chunk = static_cast<const uint8_t*>(hidden) + (size_t)t0 * d * 2;
+        if ((d3 ? make_map_mn3d(ctx, &map_h_mn, h_chunk, (uint64_t)rows, (uint64_t)d, (uint64_t)d, BN / 64)
+                : make_map(ctx, &map_h_mn, h_chunk, (uint64_t)rows, (uint64_t)d, BK)) != ARROL_OK)
             return ARROL_ERR_CUDA;
 
         DzParams zp;
@@ -530,14 +536,14 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
         dz_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h_k, map_w_k, zp);
 
         GemmParams gh;    // dH[chunk] = dZ . W
-        gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0; gh.k_is_tokens = 0;
+        gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0; gh.k_is_tokens = 0; gh.a3d = 0; gh.b3d = d3;
         gh.d_T = d_T; gh.T_max = T_max; gh.t0 = t0; gh.d_status = ctx->d_status;
         const int64_t gh_items = (int64_t)((rows + BM - 1) / BM) * ((d + BN - 1) / BN);
         gemm_kernel<false, true><<<(unsigned)(gh_items < ctx->sm_count ? gh_items : ctx->sm_count), NUM_THREADS,
                                    SMEM_BYTES, s>>>(map_dz_k, map_w_mn, map_w_mn, gh);
         tail_block_kernel<<<64, 256, 0, s>>>(static_cast<const uint16_t*>(hidden), d, d_T, T_max, t0, Htail);
         GemmParams gw;    // dW += dZ^T . H[chunk]
-        gw.M = V; gw.N = d; gw.K = (int)rows; gw.C = dW; gw.ldc = d; gw.accumulate = 1; gw.k_is_tokens = 1;
+        gw.M = V; gw.N = d; gw.K = (int)rows; gw.C = dW; gw.ldc = d; gw.accumulate = 1; gw.k_is_tokens = 1; gw.a3d = v3; gw.b3d = d3;
         gw.d_T = d_T; gw.T_max = T_max; gw.t0 = t0; gw.d_status = ctx->d_status;
         const int64_t gw_items = (int64_t)((V + BM - 1) / BM) * ((d + BN - 1) / BN);
         gemm_kernel<true, true><<<(unsigned)(gw_items < ctx->sm_count ? gw_items : ctx->sm_count), NUM_THREADS,

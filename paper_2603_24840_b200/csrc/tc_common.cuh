@@ -51,6 +51,12 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)) : "memory");
+}
+
 __device__ __forceinline__ void tcgen05_alloc(uint32_t* smem_result, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
                  "r"(cols) : "memory");
@@ -173,6 +179,21 @@ int make_map_ld(arrol_ctx* ctx, CUtensorMap* map, const void* base, uint64_t row
     const cuuint32_t elem_strides[2] = {1, 1};
     CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
         map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem_strides,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? ARROL_OK : ARROL_ERR_CUDA;
+}
+// MN-major view of [rows, cols] bf16 (rows `ld` elements apart, cols a multiple of 64) for one copy per stage:
+// dimensions (64 contiguous elements, rows, cols / 64 blocks of 128 bytes), box 64 x 64 rows x `box_blocks`, so a
+// stage receives `box_blocks` blocks of [64 rows x 128 bytes], each 128-byte swizzled, 8 KB apart.
+int make_map_mn3d(arrol_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint64_t ld,
+                  uint32_t box_blocks) {
+    const cuuint64_t dims[3] = {64, rows, cols / 64};
+    const cuuint64_t strides[2] = {ld * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)BK, box_blocks};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled)(
+        map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem_strides,
         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? ARROL_OK : ARROL_ERR_CUDA;
