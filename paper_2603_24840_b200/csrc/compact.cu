@@ -14,6 +14,8 @@
 namespace {
 
 constexpr int SCAN_THREADS = 1024;
+constexpr int SCAN_ITEMS = 4;      // consecutive rollouts per thread and pass: N <= 4096 is one pass
+constexpr int SCAN_GROUPS = SCAN_THREADS * SCAN_ITEMS / 4 + 2;   // groups of size >= 4 that one pass can touch
 
 __global__ void __launch_bounds__(SCAN_THREADS)
 scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ lengths, int N, int G,
@@ -24,16 +26,60 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     __shared__ int64_t warp_tok[32];
     __shared__ int32_t carry_cnt;
     __shared__ int64_t carry_tok;
+    // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them); den < 0: advantage 0
+    __shared__ double g_mean[SCAN_GROUPS], g_den[SCAN_GROUPS];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const bool shared_stats = G >= 4;
     if (threadIdx.x == 0) { carry_cnt = 0; carry_tok = 0; cu_seqlens[0] = 0; }
     __syncthreads();
 
-    for (int base = 0; base < N; base += SCAN_THREADS) {
-        const int i = base + threadIdx.x;
-        const bool kept = (i < N) && keep[i] != 0;
-        int32_t c = kept ? 1 : 0;
-        int64_t t = kept ? (int64_t)max(lengths[i], 0) : 0;
-        // inclusive scan inside the warp
+    // statistics over the kept rollouts of a group (Section 3, on survivors): sums in index order, fp64
+    auto group_stats = [&](int g, double& mean, double& den) {
+        const int g0 = g * G;
+        const int g1 = min(g0 + G, N);
+        // the loads do not depend on the flags, so they overlap; adding 0.0 for a pruned rollout changes nothing
+        int n = 0;
+        double sum = 0.0;
+#pragma unroll 4
+        for (int r = g0; r < g1; ++r) {
+            const bool k = keep[r] != 0;
+            const double v = (double)rewards[r];
+            sum += k ? v : 0.0;
+            n += k ? 1 : 0;
+        }
+        mean = sum / (double)n;
+        double ss = 0.0;
+#pragma unroll 4
+        for (int r = g0; r < g1; ++r) {
+            const bool k = keep[r] != 0;
+            const double dv = (double)rewards[r] - mean;
+            ss += k ? dv * dv : 0.0;
+        }
+        den = (n - ddof > 0) ? sqrt(ss / (double)(n - ddof)) + eps : -1.0;
+    };
+
+    for (int base = 0; base < N; base += SCAN_THREADS * SCAN_ITEMS) {
+        const int i0 = base + threadIdx.x * SCAN_ITEMS;
+        bool kept[SCAN_ITEMS];
+        int64_t len[SCAN_ITEMS];
+        int32_t c = 0;
+        int64_t t = 0;
+#pragma unroll
+        for (int u = 0; u < SCAN_ITEMS; ++u) {     // all loads of the pass are issued before the first use
+            const int i = i0 + u;
+            kept[u] = (i < N) && keep[i] != 0;
+            len[u] = kept[u] ? (int64_t)max(lengths[i], 0) : 0;
+        }
+        const int g_lo = base / G;
+        if (shared_stats) {          // one thread per group of this pass; visible after the scan's first barrier
+            const int g_hi = (min(N, base + SCAN_THREADS * SCAN_ITEMS) - 1) / G;
+            for (int gi = threadIdx.x; gi <= g_hi - g_lo; gi += SCAN_THREADS) group_stats(g_lo + gi, g_mean[gi], g_den[gi]);
+        }
+#pragma unroll
+        for (int u = 0; u < SCAN_ITEMS; ++u) { c += kept[u] ? 1 : 0; t += len[u]; }
+        const int32_t own_c = c;
+        const int64_t own_t = t;
+        // inclusive scan of the per-thread totals inside the warp
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int32_t oc = __shfl_up_sync(0xffffffffu, c, o);
@@ -55,26 +101,21 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
             warp_tok[lane] = wt;
         }
         __syncthreads();
-        const int32_t cnt_before = carry_cnt + (wid ? warp_cnt[wid - 1] : 0);
-        const int64_t tok_before = carry_tok + (wid ? warp_tok[wid - 1] : 0);
-        if (kept) {
-            const int32_t pos = cnt_before + c - 1;        // survivor ordinal
+        int32_t pos = carry_cnt + (wid ? warp_cnt[wid - 1] : 0) + (c - own_c);   // survivors before this thread's items
+        int64_t tok = carry_tok + (wid ? warp_tok[wid - 1] : 0) + (t - own_t);
+#pragma unroll
+        for (int u = 0; u < SCAN_ITEMS; ++u) {
+            if (!kept[u]) continue;
+            const int i = i0 + u;
+            tok += len[u];
             survivor_idx[pos] = i;
-            cu_seqlens[pos + 1] = tok_before + t;
-            // statistics over the kept rollouts of this rollout's group (Section 3, on survivors)
-            const int g0 = (i / G) * G;
-            const int g1 = min(g0 + G, N);
-            int n = 0;
-            double sum = 0.0;
-            for (int r = g0; r < g1; ++r)
-                if (keep[r]) { sum += (double)rewards[r]; ++n; }
-            const double mean = sum / (double)n;
-            double ss = 0.0;
-            for (int r = g0; r < g1; ++r)
-                if (keep[r]) { const double dv = (double)rewards[r] - mean; ss += dv * dv; }
-            double a = 0.0;
-            if (n - ddof > 0) a = ((double)rewards[i] - mean) / (sqrt(ss / (double)(n - ddof)) + eps);
+            cu_seqlens[pos + 1] = tok;
+            double mean, den;
+            if (shared_stats) { mean = g_mean[i / G - g_lo]; den = g_den[i / G - g_lo]; }
+            else group_stats(i / G, mean, den);
+            const double a = den < 0.0 ? 0.0 : ((double)rewards[i] - mean) / den;
             adv[pos] = (float)a;
+            ++pos;
         }
         __syncthreads();
         if (threadIdx.x == 0) { carry_cnt += warp_cnt[31]; carry_tok += warp_tok[31]; }
@@ -179,6 +220,41 @@ gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_
     }
 }
 
+// Per-token outputs without a payload plane (token ids, survivor ordinal, advantage): one block per survivor walks
+// its run of tokens with coalesced 4-byte accesses, so nothing has to be searched.  Blocks past S return at once.
+constexpr int TOKENS_THREADS = 128;
+__global__ void __launch_bounds__(TOKENS_THREADS)
+gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_seqlens,
+                     const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
+                     const int32_t* __restrict__ src_tokens, const float* __restrict__ adv, int64_t capacity,
+                     int32_t* __restrict__ dst_tokens, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
+    const int S = (int)d_num[0];
+    if (d_num[1] > capacity) return;                       // capacity overflow was recorded by the scan kernel
+    for (int s = blockIdx.x; s < S; s += gridDim.x) {
+        const int64_t c0 = __ldg(cu_seqlens + s);
+        const int len = (int)(__ldg(cu_seqlens + s + 1) - c0);
+        const int64_t src0 = __ldg(src_tok_off + __ldg(survivor_idx + s));
+        const float a = __ldg(adv + s);
+        for (int t0 = threadIdx.x; t0 < len; t0 += 4 * TOKENS_THREADS) {
+            int32_t tok[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int t = t0 + u * TOKENS_THREADS;
+                if (dst_tokens && t < len) tok[u] = __ldg(src_tokens + src0 + t);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int t = t0 + u * TOKENS_THREADS;
+                if (t < len) {
+                    if (dst_tokens) dst_tokens[c0 + t] = tok[u];
+                    if (tok_seq) tok_seq[c0 + t] = s;
+                    if (tok_adv) tok_adv[c0 + t] = a;
+                }
+            }
+        }
+    }
+}
+
 }  // namespace
 
 extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths,
@@ -211,13 +287,19 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
 
     const int vec_per_row = src_rows ? row_bytes / 16 : 0;
-    int tile_rows = MAX_TILE_ROWS;
-    if (vec_per_row > 0) {
-        // as many whole rows as fit one 32 KB pass (rows larger than that take several passes each)
-        tile_rows = BATCH_VECS / vec_per_row;
-        if (tile_rows < 1) tile_rows = 1;
-        if (tile_rows > MAX_TILE_ROWS) tile_rows = MAX_TILE_ROWS;
+    if (vec_per_row == 0) {
+        int64_t blocks = N < (int64_t)ctx->sm_count * 16 ? N : (int64_t)ctx->sm_count * 16;
+        gather_tokens_kernel<<<(unsigned)blocks, TOKENS_THREADS, 0, s>>>(
+            d_num, cu_seqlens, survivor_idx, src_tok_off, src_tokens, adv, dst_capacity_tokens, dst_tokens, tok_adv,
+            tok_seq);
+        ctx->launches += 1;
+        ARROL_CUDA_OK(cudaGetLastError());
+        return ARROL_OK;
     }
+    // as many whole rows as fit one 32 KB pass (rows larger than that take several passes each)
+    int tile_rows = BATCH_VECS / vec_per_row;
+    if (tile_rows < 1) tile_rows = 1;
+    if (tile_rows > MAX_TILE_ROWS) tile_rows = MAX_TILE_ROWS;
     if ((int64_t)tile_rows * vec_per_row > INT32_MAX) return ARROL_ERR_UNSUPPORTED;
     const int64_t max_tiles = (dst_capacity_tokens + tile_rows - 1) / tile_rows;
     // Exactly one wave: every block owns an equal contiguous share of the destination, so a partial second wave
