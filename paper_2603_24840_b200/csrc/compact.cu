@@ -28,22 +28,30 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     __shared__ int64_t carry_tok;
     // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them); den < 0: advantage 0
     __shared__ double g_mean[SCAN_GROUPS], g_den[SCAN_GROUPS];
+    // the pass's keep flags and rewards, staged once so that the statistics and the advantages read shared memory
+    __shared__ float s_rew[SCAN_THREADS * SCAN_ITEMS];
+    __shared__ uint8_t s_keep[SCAN_THREADS * SCAN_ITEMS];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const bool shared_stats = G >= 4;
     if (threadIdx.x == 0) { carry_cnt = 0; carry_tok = 0; cu_seqlens[0] = 0; }
     __syncthreads();
 
     // statistics over the kept rollouts of a group (Section 3, on survivors): sums in index order, fp64
-    auto group_stats = [&](int g, double& mean, double& den) {
+    constexpr int PASS = SCAN_THREADS * SCAN_ITEMS;
+    auto group_stats = [&](int g, int base, double& mean, double& den) {
         const int g0 = g * G;
         const int g1 = min(g0 + G, N);
-        // the loads do not depend on the flags, so they overlap; adding 0.0 for a pruned rollout changes nothing
+        // members inside the staged pass come from shared memory, a group that straddles its edge reads the rest
+        // from global memory; the loads do not depend on the flags, so they overlap; adding 0.0 for a pruned
+        // rollout changes nothing
+        auto flag = [&](int r) { return (unsigned)(r - base) < (unsigned)PASS ? s_keep[r - base] != 0 : keep[r] != 0; };
+        auto rew = [&](int r) { return (unsigned)(r - base) < (unsigned)PASS ? s_rew[r - base] : rewards[r]; };
         int n = 0;
         double sum = 0.0;
 #pragma unroll 4
         for (int r = g0; r < g1; ++r) {
-            const bool k = keep[r] != 0;
-            const double v = (double)rewards[r];
+            const bool k = flag(r);
+            const double v = (double)rew(r);
             sum += k ? v : 0.0;
             n += k ? 1 : 0;
         }
@@ -51,29 +59,38 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
         double ss = 0.0;
 #pragma unroll 4
         for (int r = g0; r < g1; ++r) {
-            const bool k = keep[r] != 0;
-            const double dv = (double)rewards[r] - mean;
+            const bool k = flag(r);
+            const double dv = (double)rew(r) - mean;
             ss += k ? dv * dv : 0.0;
         }
         den = (n - ddof > 0) ? sqrt(ss / (double)(n - ddof)) + eps : -1.0;
     };
 
-    for (int base = 0; base < N; base += SCAN_THREADS * SCAN_ITEMS) {
+    for (int base = 0; base < N; base += PASS) {
         const int i0 = base + threadIdx.x * SCAN_ITEMS;
         bool kept[SCAN_ITEMS];
         int64_t len[SCAN_ITEMS];
         int32_t c = 0;
         int64_t t = 0;
+        // one round of coalesced loads: flags and rewards of the pass into shared memory, lengths into registers
+        for (int e = threadIdx.x; e < PASS; e += SCAN_THREADS) {
+            const int i = base + e;
+            s_keep[e] = i < N ? keep[i] : (uint8_t)0;
+            s_rew[e] = i < N ? rewards[i] : 0.f;
+        }
 #pragma unroll
-        for (int u = 0; u < SCAN_ITEMS; ++u) {     // all loads of the pass are issued before the first use
-            const int i = i0 + u;
-            kept[u] = (i < N) && keep[i] != 0;
-            len[u] = kept[u] ? (int64_t)max(lengths[i], 0) : 0;
+        for (int u = 0; u < SCAN_ITEMS; ++u) len[u] = (i0 + u < N) ? (int64_t)max(lengths[i0 + u], 0) : 0;
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < SCAN_ITEMS; ++u) {
+            kept[u] = s_keep[threadIdx.x * SCAN_ITEMS + u] != 0;
+            if (!kept[u]) len[u] = 0;
         }
         const int g_lo = base / G;
         if (shared_stats) {          // one thread per group of this pass; visible after the scan's first barrier
-            const int g_hi = (min(N, base + SCAN_THREADS * SCAN_ITEMS) - 1) / G;
-            for (int gi = threadIdx.x; gi <= g_hi - g_lo; gi += SCAN_THREADS) group_stats(g_lo + gi, g_mean[gi], g_den[gi]);
+            const int g_hi = (min(N, base + PASS) - 1) / G;
+            for (int gi = threadIdx.x; gi <= g_hi - g_lo; gi += SCAN_THREADS)
+                group_stats(g_lo + gi, base, g_mean[gi], g_den[gi]);
         }
 #pragma unroll
         for (int u = 0; u < SCAN_ITEMS; ++u) { c += kept[u] ? 1 : 0; t += len[u]; }
@@ -112,8 +129,8 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
             cu_seqlens[pos + 1] = tok;
             double mean, den;
             if (shared_stats) { mean = g_mean[i / G - g_lo]; den = g_den[i / G - g_lo]; }
-            else group_stats(i / G, mean, den);
-            const double a = den < 0.0 ? 0.0 : ((double)rewards[i] - mean) / den;
+            else group_stats(i / G, base, mean, den);
+            const double a = den < 0.0 ? 0.0 : ((double)s_rew[i - base] - mean) / den;
             adv[pos] = (float)a;
             ++pos;
         }
