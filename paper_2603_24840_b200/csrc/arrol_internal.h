@@ -56,6 +56,32 @@ struct ArrolDeviceGuard {
     int cur = -1;
 };
 
+#ifdef __CUDACC__
+// Programmatic dependent launch for the short kernels of the prune step (score -> select -> scan -> gather), which
+// run back to back on one stream and last a few microseconds each: a kernel launched with arrol_launch_pdl may
+// start while its predecessor is still running, sets up (shared memory, barriers, tensor-map prefetch) and then
+// blocks in pdl_wait() until the predecessor has completed and its writes are visible.  Every such kernel calls
+// pdl_launch_dependents() at its top and touches global memory only after pdl_wait().
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t arrol_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                             Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // score.cu: MLP tile pass with optional pre-activation output; partial is [ceil(h / ARROL_MLP_TH)][N].
 int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index, int N,
                              const arrol_head* head, float* partial, float* u_out, cudaStream_t s);

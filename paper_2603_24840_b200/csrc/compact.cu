@@ -33,6 +33,8 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     __shared__ uint8_t s_keep[SCAN_THREADS * SCAN_ITEMS];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const bool shared_stats = G >= 4;
+    pdl_launch_dependents();
+    pdl_wait();
     if (threadIdx.x == 0) { carry_cnt = 0; carry_tok = 0; cu_seqlens[0] = 0; }
     __syncthreads();
 
@@ -182,6 +184,8 @@ gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_
               uint4* __restrict__ dst_rows, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
     __shared__ int64_t src_row_of[MAX_TILE_ROWS];
     __shared__ int s_first[2];               // survivor of the first row of the current / next tile
+    pdl_launch_dependents();
+    pdl_wait();
     const int S = (int)d_num[0];
     const int64_t T = d_num[1];
     if (T > capacity || S <= 0 || T <= 0) return;      // capacity overflow was recorded by the scan kernel
@@ -245,6 +249,8 @@ gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restric
                      const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
                      const int32_t* __restrict__ src_tokens, const float* __restrict__ adv, int64_t capacity,
                      int32_t* __restrict__ dst_tokens, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int S = (int)d_num[0];
     if (d_num[1] > capacity) return;                       // capacity overflow was recorded by the scan kernel
     for (int s = blockIdx.x; s < S; s += gridDim.x) {
@@ -295,22 +301,20 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     ArrolDeviceGuard guard(ctx->device);
     if (!guard.ok) return ARROL_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
-    scan_adv_kernel<<<1, SCAN_THREADS, 0, s>>>(keep, lengths, N, G, rewards, (double)eps, ddof,
-                                               dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
-                                               ctx->d_status);
+    ARROL_CUDA_OK(arrol_launch_pdl(scan_adv_kernel, dim3(1), dim3(SCAN_THREADS), 0, s, keep, lengths, N, G, rewards,
+                                   (double)eps, ddof, dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
+                                   ctx->d_status));
     ctx->launches += 1;
-    ARROL_CUDA_OK(cudaGetLastError());
     const bool any_token_output = dst_tokens || dst_rows || tok_adv || tok_seq;
     if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
 
     const int vec_per_row = src_rows ? row_bytes / 16 : 0;
     if (vec_per_row == 0) {
         int64_t blocks = N < (int64_t)ctx->sm_count * 16 ? N : (int64_t)ctx->sm_count * 16;
-        gather_tokens_kernel<<<(unsigned)blocks, TOKENS_THREADS, 0, s>>>(
-            d_num, cu_seqlens, survivor_idx, src_tok_off, src_tokens, adv, dst_capacity_tokens, dst_tokens, tok_adv,
-            tok_seq);
+        ARROL_CUDA_OK(arrol_launch_pdl(gather_tokens_kernel, dim3((unsigned)blocks), dim3(TOKENS_THREADS), 0, s, d_num,
+                                       cu_seqlens, survivor_idx, src_tok_off, src_tokens, adv, dst_capacity_tokens,
+                                       dst_tokens, tok_adv, tok_seq));
         ctx->launches += 1;
-        ARROL_CUDA_OK(cudaGetLastError());
         return ARROL_OK;
     }
     // as many whole rows as fit one 32 KB pass (rows larger than that take several passes each)
@@ -327,11 +331,10 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     int64_t blocks = (int64_t)ctx->sm_count * resident;
     if (blocks > max_tiles) blocks = max_tiles;
     if (blocks < 1) blocks = 1;
-    gather_kernel<<<(unsigned)blocks, GATHER_THREADS, 0, s>>>(
-        d_num, cu_seqlens, survivor_idx, src_tok_off, src_tokens, static_cast<const uint4*>(src_rows),
-        vec_per_row, adv, dst_capacity_tokens, tile_rows, dst_tokens, static_cast<uint4*>(dst_rows), tok_adv,
-        tok_seq);
+    ARROL_CUDA_OK(arrol_launch_pdl(gather_kernel, dim3((unsigned)blocks), dim3(GATHER_THREADS), 0, s, d_num, cu_seqlens,
+                                   survivor_idx, src_tok_off, src_tokens, static_cast<const uint4*>(src_rows),
+                                   vec_per_row, adv, dst_capacity_tokens, tile_rows, dst_tokens,
+                                   static_cast<uint4*>(dst_rows), tok_adv, tok_seq));
     ctx->launches += 1;
-    ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
 }

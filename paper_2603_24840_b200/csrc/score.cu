@@ -62,6 +62,8 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
                     int d, const T* __restrict__ w, const T* __restrict__ bias, int B,
                     const float* __restrict__ q_lut, float* score, float* prob, int32_t* bin, float* q) {
     constexpr int VN = Vec16<T>::N;
+    pdl_launch_dependents();
+    pdl_wait();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= N) return;
@@ -282,9 +284,9 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
     if (head->h == 0) {
         const int warps_per_block = 4;
         const int blocks = (N + warps_per_block - 1) / warps_per_block;
-        score_linear_kernel<T><<<blocks, 32 * warps_per_block, 0, s>>>(
-            hid, row_stride, row_index, N, head->d, static_cast<const T*>(head->W1),
-            static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q);
+        ARROL_CUDA_OK(arrol_launch_pdl(score_linear_kernel<T>, dim3(blocks), dim3(32 * warps_per_block), 0, s, hid,
+                                       row_stride, row_index, N, head->d, static_cast<const T*>(head->W1),
+                                       static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q));
         ctx->launches += 1;
     } else {
         if constexpr (sizeof(T) == 2) {

@@ -37,6 +37,8 @@ constexpr size_t S_SMEM_BYTES = (size_t)S_STAGES * S_STAGE_BYTES + 1024 + S_TAIL
 __global__ void __launch_bounds__(128)
 pack_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index,
                  int N, int d, __nv_bfloat16* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (i >= N) return;
@@ -104,6 +106,8 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         tcgen05_alloc(tmem_slot, S_TMEM_COLS);
         tcgen05_relinquish();
     }
+    pdl_launch_dependents();
+    pdl_wait();                  // set-up above overlaps the previous kernel; global memory is read from here on
     if (warp >= 2 * S_PAIRS) {   // the tile's slice of b1 and w2, zero past h so that padded columns add nothing
         const int e = threadIdx.x - 2 * S_PAIRS * 32;
         if (e < SBN) {
@@ -248,8 +252,9 @@ int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_
     const void* x = hidden;
     int64_t ld = row_stride;
     if (row_index) {
-        pack_rows_kernel<<<(N + 3) / 4, 128, 0, s>>>(static_cast<const __nv_bfloat16*>(hidden), row_stride, row_index,
-                                                     N, d, static_cast<__nv_bfloat16*>(ctx->d_pack));
+        ARROL_CUDA_OK(arrol_launch_pdl(pack_rows_kernel, dim3((N + 3) / 4), dim3(128), 0, s,
+                                       static_cast<const __nv_bfloat16*>(hidden), row_stride, row_index, N, d,
+                                       static_cast<__nv_bfloat16*>(ctx->d_pack)));
         ctx->launches += 1;
         x = ctx->d_pack;
         ld = d;
@@ -277,8 +282,7 @@ int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_
     ARROL_CUDA_OK(cudaFuncSetAttribute(score_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)S_SMEM_BYTES));
     dim3 grid(m_tiles, h_tiles);
-    score_mlp_tc_kernel<<<grid, S_THREADS, S_SMEM_BYTES, s>>>(map_x, map_w, p);
+    ARROL_CUDA_OK(arrol_launch_pdl(score_mlp_tc_kernel, grid, dim3(S_THREADS), S_SMEM_BYTES, s, map_x, map_w, p));
     ctx->launches += 1;
-    ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
 }

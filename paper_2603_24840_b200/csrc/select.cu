@@ -26,6 +26,8 @@ __device__ __forceinline__ double shfl_xor_double(double v, int mask, int width)
 
 __global__ void __launch_bounds__(128)
 select_kernel(const float* __restrict__ q, int P, int G, int K, double rho, int seg, uint8_t* __restrict__ keep) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int groups_per_warp = 32 / seg;
@@ -75,9 +77,8 @@ extern "C" int arrol_select(arrol_ctx* ctx, const float* q, int32_t P, int32_t G
     const int warps_per_block = 4;
     ArrolDeviceGuard guard(ctx->device);
     if (!guard.ok) return ARROL_ERR_CUDA;
-    select_kernel<<<(warps + warps_per_block - 1) / warps_per_block, 32 * warps_per_block, 0,
-                    (cudaStream_t)stream>>>(q, P, G, K, rho, seg, keep);
+    ARROL_CUDA_OK(arrol_launch_pdl(select_kernel, dim3((warps + warps_per_block - 1) / warps_per_block),
+                                   dim3(32 * warps_per_block), 0, (cudaStream_t)stream, q, P, G, K, rho, seg, keep));
     ctx->launches += 1;
-    ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
 }
