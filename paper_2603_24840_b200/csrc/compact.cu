@@ -15,6 +15,7 @@ namespace {
 
 constexpr int SCAN_THREADS = 1024;
 constexpr int SCAN_ITEMS = 4;      // consecutive rollouts per thread and pass: N <= 4096 is one pass
+constexpr int SCAN_INV = 65;
 constexpr int SCAN_GROUPS = SCAN_THREADS * SCAN_ITEMS / 4 + 2;   // groups of size >= 4 that one pass can touch
 
 __global__ void __launch_bounds__(SCAN_THREADS)
@@ -26,11 +27,12 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     __shared__ int64_t warp_tok[32];
     __shared__ int32_t carry_cnt;
     __shared__ int64_t carry_tok;
-    // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them); den < 0: advantage 0
-    __shared__ double g_mean[SCAN_GROUPS], g_den[SCAN_GROUPS];
+    // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them)
+    __shared__ double g_mean[SCAN_GROUPS], g_den[SCAN_GROUPS];     // mean, 1 / (std + eps)
     // the pass's keep flags and rewards, staged once so that the statistics and the advantages read shared memory
     __shared__ float s_rew[SCAN_THREADS * SCAN_ITEMS];
     __shared__ uint8_t s_keep[SCAN_THREADS * SCAN_ITEMS];
+    __shared__ double s_inv[SCAN_INV];             // 1 / count for the small counts
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const bool shared_stats = G >= 4;
     pdl_launch_dependents();
@@ -40,7 +42,12 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
 
     // statistics over the kept rollouts of a group (Section 3, on survivors): sums in index order, fp64
     constexpr int PASS = SCAN_THREADS * SCAN_ITEMS;
-    auto group_stats = [&](int g, int base, double& mean, double& den) {
+    // Statistics of group g over its kept rollouts: mean and 1 / (std + eps), in fp64.  A double-precision division
+    // or square root costs this one-block kernel about half a microsecond each, so the reciprocals of the small
+    // counts come from a table and sqrt / reciprocal are Newton steps from single-precision seeds (relative error
+    // below 1e-15 after two steps); values outside the single-precision range take the plain operations.
+    // inv_den = 0 (advantage exactly 0) when fewer than ddof + 1 rollouts are kept or all kept rewards are equal.
+    auto group_stats = [&](int g, int base, double& mean, double& inv_den) {
         const int g0 = g * G;
         const int g1 = min(g0 + G, N);
         // members inside the staged pass come from shared memory, a group that straddles its edge reads the rest
@@ -50,14 +57,19 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
         auto rew = [&](int r) { return (unsigned)(r - base) < (unsigned)PASS ? s_rew[r - base] : rewards[r]; };
         int n = 0;
         double sum = 0.0;
+        float first = 0.f;
+        bool all_equal = true;
 #pragma unroll 4
         for (int r = g0; r < g1; ++r) {
             const bool k = flag(r);
-            const double v = (double)rew(r);
-            sum += k ? v : 0.0;
+            const float v = rew(r);
+            if (k && n == 0) first = v;
+            all_equal = all_equal && (!k || v == first);
+            sum += k ? (double)v : 0.0;
             n += k ? 1 : 0;
         }
-        mean = sum / (double)n;
+        auto recip_count = [&](int c) { return c < SCAN_INV ? s_inv[c] : 1.0 / (double)c; };
+        mean = n > 0 ? sum * recip_count(n) : 0.0;
         double ss = 0.0;
 #pragma unroll 4
         for (int r = g0; r < g1; ++r) {
@@ -65,8 +77,33 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
             const double dv = (double)rew(r) - mean;
             ss += k ? dv * dv : 0.0;
         }
-        den = (n - ddof > 0) ? sqrt(ss / (double)(n - ddof)) + eps : -1.0;
+        inv_den = 0.0;
+        if (n - ddof > 0 && !all_equal) {
+            const double var = ss * recip_count(n - ddof);
+            double sd;
+            const float varf = (float)var;
+            if (varf > 1e-30f && varf < 1e30f) {
+                double y = (double)rsqrtf(varf);
+                y = y * (1.5 - 0.5 * var * y * y);
+                y = y * (1.5 - 0.5 * var * y * y);
+                sd = var * y;
+            } else {
+                sd = sqrt(var);
+            }
+            const double den = sd + eps;
+            const float denf = (float)den;
+            if (denf > 1e-30f && denf < 1e30f) {
+                double x = (double)(1.0f / denf);
+                x = x * (2.0 - den * x);
+                x = x * (2.0 - den * x);
+                inv_den = x;
+            } else {
+                inv_den = 1.0 / den;
+            }
+        }
     };
+
+    if (threadIdx.x >= 1 && threadIdx.x < SCAN_INV) s_inv[threadIdx.x] = 1.0 / (double)threadIdx.x;   // before the first barrier below
 
     for (int base = 0; base < N; base += PASS) {
         const int i0 = base + threadIdx.x * SCAN_ITEMS;
@@ -132,7 +169,7 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
             double mean, den;
             if (shared_stats) { mean = g_mean[i / G - g_lo]; den = g_den[i / G - g_lo]; }
             else group_stats(i / G, base, mean, den);
-            const double a = den < 0.0 ? 0.0 : ((double)s_rew[i - base] - mean) / den;
+            const double a = ((double)s_rew[i - base] - mean) * den;      // den holds 1 / (std + eps), or 0
             adv[pos] = (float)a;
             ++pos;
         }
