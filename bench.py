@@ -281,6 +281,31 @@ def run_ours(args, w):
         b.record(stream)
         torch.cuda.synchronize()
         prune_us[label] = a.elapsed_time(b) / reps * 1e3
+    # the same token-only step replayed from a captured CUDA graph: the four to five launches cost the host one call,
+    # so this is the device-side duration of the chain (the eager figure above includes host launch time)
+    try:
+        step_args = pr.prune_step_args(with_rows=False)
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            B.arrol_prune_step(pr.ctx, step_args)              # warm-up on the capture stream
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            B.arrol_prune_step(pr.ctx, step_args)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        reps = max(K, 20)
+        a.record(stream)
+        for _ in range(reps):
+            graph.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        prune_us["tokens_only_graph"] = a.elapsed_time(b) / reps * 1e3
+        del graph
+    except RuntimeError as exc:
+        print("graph replay of the prune step skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
 
     # scoring kernel on its own: the linear head streamed over every source row (HBM-bound: d*e bytes per row);
     # the MLP head on the workload's own N rollouts (2*d*h flops per row, on the tensor cores for bf16 heads)

@@ -159,7 +159,10 @@ int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab,
 
 /* ---- Prune step in one call (Algorithm 1: quality check at the detection length, filter, re-batch) ----------
  * arrol_score_partial -> arrol_select -> arrol_compact issued back to back on `stream` with N = P * G; every field
- * has the meaning, layout and nullability of the argument of the same name in those calls.  Asynchronous. */
+ * has the meaning, layout and nullability of the argument of the same name in those calls.  Asynchronous.
+ * The kernels are launched with programmatic stream serialization (each sets up while its predecessor finishes and
+ * reads global memory only after the predecessor has completed).  The call allocates nothing and never
+ * synchronises, so it may be captured into a CUDA graph and replayed. */
 typedef struct arrol_prune_step_args {
     /* scoring */
     const void* hidden;
