@@ -29,6 +29,10 @@ constexpr int EPI_WARPS = 8;            // two warps per tensor-memory lane quar
 constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int EPI_PIECES = BN / 32 / (EPI_WARPS / 4);   // 32-column pieces per epilogue warp and accumulator
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+// dz_kernel: one 32-row x 128-byte staging tile per epilogue warp behind the barrier block (1 KB), 1024-byte aligned
+constexpr int DZ_STAGE_TILE = 32 * 128;
+constexpr size_t DZ_STAGE_OFFSET = (size_t)STAGES * STAGE_BYTES + 1024;
+constexpr size_t DZ_SMEM_BYTES = DZ_STAGE_OFFSET + (size_t)EPI_WARPS * DZ_STAGE_TILE + 1024;
 constexpr int TC = 74 * BM;      // tokens per chunk: 74 token tiles, so that TC/128 x d/256 tiles fill 148 SMs evenly
 
 struct PipeSmem {
@@ -208,9 +212,11 @@ struct DzParams {
 };
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, const DzParams p) {
+dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
+          const __grid_constant__ CUtensorMap map_dz, const DzParams p) {
     extern __shared__ uint8_t smem_raw[];
     const PipeSmem ps = carve_smem(smem_raw);
+    uint8_t* dz_stage = ps.stage_a + DZ_STAGE_OFFSET;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t T = live_tokens(p.d_T, p.T_max);
     if (p.t0 >= T) return;                                  // chunk past the live tokens (uniform for the grid)
@@ -278,19 +284,22 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                     y = -1;
                 }
             }
-            __nv_bfloat16* zrow = p.dZ + (int64_t)row_in_chunk * p.ldz;
+            // dz leaves through shared memory: the warp's 32 rows x 64 columns (two pieces, 128 bytes per row, 128-byte
+            // swizzle) are staged and written by one TMA tile store, i.e. in whole 128-byte lines; columns past V are
+            // clipped by the copy.  (16-byte stores straight from the registers touch 32 lines per instruction and
+            // cost the kernel 14 %.)
+            uint8_t* stg = dz_stage + (size_t)(warp - 2) * DZ_STAGE_TILE;
+            const int row0 = m_tile * BM + quarter * 32;
             for (int c = c0; c < c1 && ok; ++c) {
                 ok = mbar_wait(&ps.acc_full[acc], acc_phase, ps.abort_flag);
                 ok = __all_sync(0xffffffffu, ok) != 0;
                 if (!ok) break;
                 tcgen05_fence_after();
                 // Two register buffers: the tensor-memory load of piece i + 1 is in flight while piece i is turned
-                // into dz and stored.
+                // into dz and staged.
                 const uint32_t tacc = tmem_base + lane_addr + acc * BN;
-                auto emit = [&](const uint32_t (&raw)[32], int piece) {
+                auto to_dz = [&](const uint32_t (&raw)[32], int piece, uint32_t (&packed)[16]) {
                     const int pc0 = c * BN + piece * 32;
-                    if (pc0 >= p.V) return;
-                    uint32_t packed[16];
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
                         // dz = coef ([v = y] - 2^(z log2e - lse log2e)); coef = 0 for rows that carry no gradient
@@ -302,21 +311,13 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                         const __nv_bfloat162 h2 = __floats2bfloat162_rn(d0, d1);
                         packed[j >> 1] = *reinterpret_cast<const uint32_t*>(&h2);
                     }
-                    const int n_valid = min(32, p.V - pc0);
-                    if (n_valid == 32) {
-                        uint4* dst = reinterpret_cast<uint4*>(zrow + pc0);
+                };
+                auto stage_piece = [&](const uint32_t (&packed)[16], int piece) {
+                    const int chunk0 = (piece & 1) * 4;               // 16-byte chunks of the 128-byte staging row
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4)
-                            dst[q4] = make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < n_valid) {
-                                const uint32_t w = packed[j >> 1];
-                                reinterpret_cast<uint16_t*>(zrow)[pc0 + j] = (uint16_t)((j & 1) ? (w >> 16) : (w & 0xffffu));
-                            }
-                        }
-                    }
+                    for (int q4 = 0; q4 < 4; ++q4)
+                        *reinterpret_cast<uint4*>(stg + lane * 128 + (((chunk0 + q4) ^ (lane & 7)) << 4)) =
+                            make_uint4(packed[4 * q4], packed[4 * q4 + 1], packed[4 * q4 + 2], packed[4 * q4 + 3]);
                 };
                 uint32_t ra[32], rb[32];
                 const int p0 = col_half * EPI_PIECES, p1 = p0 + EPI_PIECES;   // this warp's pieces of the accumulator
@@ -325,10 +326,22 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                 for (int piece = p0; piece < p1; piece += 2) {
                     tcgen05_ld_wait(ra);
                     tcgen05_ld_32x32_issue(tacc + (piece + 1) * 32, rb);
-                    emit(ra, piece);
+                    uint32_t pa[16], pb[16];
+                    to_dz(ra, piece, pa);
                     tcgen05_ld_wait(rb);
                     if (piece + 2 < p1) tcgen05_ld_32x32_issue(tacc + (piece + 2) * 32, ra);
-                    emit(rb, piece + 1);
+                    to_dz(rb, piece + 1, pb);
+                    if (lane == 0) bulk_wait_read_all();          // the previous tile store has read the staging tile
+                    __syncwarp();
+                    stage_piece(pa, piece);
+                    stage_piece(pb, piece + 1);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    const int col0 = c * BN + piece * 32;
+                    if (lane == 0 && col0 < p.V) {
+                        tma_store_2d(&map_dz, col0, row0, stg);
+                        bulk_commit_group();
+                    }
                 }
                 tcgen05_fence_before();
                 __syncwarp();
@@ -336,6 +349,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
         }
+        if (lane == 0) bulk_wait_all();       // the tile stores have completed before the block's shared memory goes
     }
     pipe_teardown(ps, tmem_base, p.d_status);
 }
@@ -490,17 +504,18 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     __nv_bfloat16* dZ = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + L.dz);
     uint16_t* Htail = reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + L.tail);
 
-    ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DZ_SMEM_BYTES));
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
 
     // tensor maps: K-major operands are fetched as [MN rows x 64 K columns] boxes; MN-major ones (the same row-major
     // storage read the other way) as one three-dimensional box per stage when the MN extent is a whole number of
     // 64-element blocks, else as one [64 K rows x 64 MN columns] box per block
-    CUtensorMap map_h_k, map_w_k, map_dz_k, map_w_mn, map_dz_mn, map_h_mn, map_h_tail;
+    CUtensorMap map_h_k, map_w_k, map_dz_k, map_dz_st, map_w_mn, map_dz_mn, map_h_mn, map_h_tail;
     if (make_map(ctx, &map_h_k, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map(ctx, &map_w_k, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map_ld(ctx, &map_dz_k, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (make_map_ld(ctx, &map_dz_st, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, 32) != ARROL_OK) return ARROL_ERR_CUDA;   // store tiles
     bool d3 = d % 64 == 0, v3 = V % 64 == 0;
     if (d3 && (make_map_mn3d(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN / 64) != ARROL_OK ||
                make_map_mn3d(ctx, &map_h_tail, Htail, (uint64_t)BK, (uint64_t)d, (uint64_t)d, BN / 64) != ARROL_OK))
@@ -533,7 +548,7 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
         zp.dZ = dZ; zp.d_status = ctx->d_status;
         int64_t grid = (int64_t)(TC / BM) * splits;
         if (grid > ctx->sm_count) grid = ctx->sm_count;
-        dz_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h_k, map_w_k, zp);
+        dz_kernel<<<(unsigned)grid, NUM_THREADS, DZ_SMEM_BYTES, s>>>(map_h_k, map_w_k, map_dz_st, zp);
 
         GemmParams gh;    // dH[chunk] = dZ . W
         gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0; gh.k_is_tokens = 0; gh.a3d = 0; gh.b3d = d3;
