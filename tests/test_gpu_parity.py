@@ -103,6 +103,13 @@ def test_mlp_head(ctx, N, d, h, dtype):
     _score_case(ctx, N, d, h, dtype, False, False, seed=N + h + 1, bias=False)
 
 
+def test_mlp_head_larger_than_the_packing_buffer_takes_the_simt_path(ctx):
+    """N * d * 2 bytes beyond the context's 64 MB row-packing buffer: the call falls back to the fp32 SIMT kernels
+    (same results); without a row index the rows are tiled in place and no packing is needed."""
+    _score_case(ctx, 8448, 4096, 64, torch.bfloat16, False, True, seed=3)     # 69 MB of scored rows, indexed
+    _score_case(ctx, 8448, 4096, 64, torch.bfloat16, True, False, seed=4)     # same size, rows in place
+
+
 def test_mlp_head_strided_rows_without_index(ctx):
     """Evenly strided rows (a column slice of a wider buffer) go to the tensor-core path without packing."""
     g = np.random.default_rng(5)
