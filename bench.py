@@ -333,6 +333,14 @@ def run_ours(args, w):
         except (RuntimeError, MemoryError) as exc:
             print("update leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
 
+    # ---- the calls around the step (reported separately; not part of `value`) ----
+    aux = None
+    if not args.skip_aux:
+        try:
+            aux = run_aux(pr, w_rank, B, torch, K)
+        except (RuntimeError, MemoryError) as exc:
+            print("aux leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
+
     # ---- e2e: host buffers through arrol_prune_rebatch_host ----
     if args.skip_e2e:
         e2e = {"ms_per_step": float("nan"), "h2d": 0, "d2h": 0}
@@ -421,6 +429,11 @@ def run_ours(args, w):
                              "achieved": upd_flops / (update["ms"] * 1e-3) / 1e12, "unit": "TFLOP/s",
                              "frac": upd_flops / (update["ms"] * 1e-3) / 1e12 / peak, "bound": "tensor",
                              "workspace_gb": update["ws_gb"]}
+        if aux is not None:
+            aux["what"] = ("calibrator update + stochastic rule on N rollouts, head training step on the N scored rows, "
+                           "rank-weighted vote over P groups, log-prob call with per-token confidence and its "
+                           "per-rollout reduction")
+            out["aux"] = aux
         if not args.no_cpu_baseline and world == 1:
             v, sample, cores, _ = oracle_step_rate(w, args.cpu_budget)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
@@ -467,6 +480,68 @@ def run_update(pr, w, B, torch, K):
         loss_ms += a.elapsed_time(mid)
     B.arrol_poll_status(pr.ctx)
     return {"ms": tot / n, "loss_ms": loss_ms / n, "ws_gb": ws_bytes / 1e9}
+
+
+def run_aux(pr, w, B, torch, K):
+    """Times the calls around the step on the workload's shapes: calibrator update + stochastic survival rule
+    (Appendix A.4), head training step, rank-weighted vote (Section 4.4), confidence variant of the log-prob call."""
+    from paper_2603_24840_b200 import calibrator as CAL, confidence as CF, headtrain as HT, voting as VT
+    dev, N = pr.dev, w.N
+    stream = torch.cuda.current_stream()
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed + 99)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3          # us
+
+    out = {}
+    reps = max(K, 20)
+    # calibrator: push the step's N (bin, reward) pairs, rebuild the table and delta; then the stochastic rule
+    cal = CAL.Calibrator(pr.ctx, w.B, 8192)
+    sp = CAL.survival(w.K / w.G, 0.5, w.rho, 0.05, 0.95)
+    u = torch.rand(N, generator=gen, device=dev)
+    keep2 = torch.empty(N, dtype=torch.uint8, device=dev)
+    out["calib_update_us"] = timed(lambda: cal.update(pr.bin, pr.rewards, sp), reps)
+    out["select_stochastic_us"] = timed(lambda: CAL.arrol_select_stochastic(pr.ctx, pr.q, u, keep2, sp, d_delta=cal.delta), reps)
+    # head training step on the N scored rows (labels = the rollouts' rewards)
+    hh = max(w.h, 1)
+    grads = {"W1": torch.empty((hh, w.d), device=dev), "b1": torch.empty(hh, device=dev)}
+    if w.h:
+        grads["w2"] = torch.empty(w.h, device=dev)
+        grads["b2"] = torch.empty(1, device=dev)
+    hloss = torch.zeros(1, dtype=torch.float64, device=dev)
+    hws = torch.empty(max(HT.arrol_head_grad_workspace(pr.ctx, N, w.d, w.h), 1), dtype=torch.uint8, device=dev)
+    out["head_grad_us"] = timed(lambda: HT.arrol_head_grad(pr.ctx, pr.hidden_score, pr.head, N, pr.rewards, grads, hloss, hws,
+                                                           row_index=pr.row_index), reps)
+    if w.h:
+        out["head_grad_tflops"] = 4.0 * N * w.d * w.h / (out["head_grad_us"] * 1e-6) / 1e12   # forward + dW1
+    # test-time vote: P groups of G scored rollouts with synthetic answers
+    answers = torch.randint(0, 6, (N,), generator=gen, device=dev, dtype=torch.int32)
+    vw = torch.empty(N, device=dev)
+    win = torch.empty(w.P, dtype=torch.int32, device=dev)
+    ww = torch.empty(w.P, device=dev)
+    if w.G <= 32:
+        out["rank_vote_us"] = timed(lambda: VT.arrol_rank_vote(pr.ctx, pr.score, answers, w.P, w.G, vw, win, ww), reps)
+    # log-prob call that also emits the per-token confidence, then the per-rollout reduction
+    conf = torch.empty(pr.cap, device=dev)
+    tconf = torch.empty(N, device=dev)
+    n = max(1, min(K, 3))
+    out["token_logprob_conf_ms"] = timed(lambda: CF.arrol_token_logprob_conf(
+        pr.ctx, pr.dst_rows, pr.W_vocab, pr.dst_tokens, pr.cap, w.d, w.V, pr.logp, conf, pr.workspace, lse=pr.lse,
+        d_T=pr.d_num[1:]), n) / 1e3
+    out["trace_confidence_us"] = timed(lambda: CF.arrol_trace_confidence(pr.ctx, conf, pr.cu_seqlens, pr.d_num, N, tconf,
+                                                                          window=2048, mode=1), reps)
+    B.arrol_poll_status(pr.ctx)
+    return out
 
 
 def auto_prompt_chunks(w):
@@ -544,6 +619,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prompt-chunks", type=int, default=0, help="0 = choose from the memory footprint")
     ap.add_argument("--skip-update", action="store_true", help="leave out the policy-update leg")
+    ap.add_argument("--skip-aux", action="store_true", help="leave out the timings of the calls around the step")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
     args = ap.parse_args()

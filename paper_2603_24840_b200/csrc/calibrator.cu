@@ -206,29 +206,38 @@ calib_update_kernel(uint8_t* state, CalibLayout L, const int32_t* __restrict__ b
     }
     __syncthreads();
 
-    // delta: 64 bisection steps on E[p](delta) = kappa, sums over bins in index order
-    if (threadIdx.x == 0) {
+    // delta: 64 bisection steps on E[p](delta) = kappa, by the first warp alone (no block barriers in the loop).  Per
+    // step the lanes form the per-bin products c_b p_b and lane 0 adds them in index order (the same rounding
+    // sequence as a plain loop: an empty bin adds exactly zero), so only the chain of B additions is serial.
+    if (wid == 0) {
+        __shared__ double prod[MAX_BINS];
         const double n = __dadd_rn(n_pos, n_neg);
         double delta = 0.0;
-        if (n > 0.0) {
+        if (n > 0.0) {                                   // uniform for the warp
             double lo = -(1.0 + lambda), hi = 1.0 + lambda;
             for (int it = 0; it < 64; ++it) {
                 const double mid = __dmul_rn(0.5, __dadd_rn(lo, hi));
                 const double base = __dadd_rn(kappa, mid);
-                double e = 0.0;
-                for (int b = 0; b < B; ++b) {
-                    if (weight[b] == 0.0) continue;           // adds exactly zero
+                for (int b = lane; b < B; b += 32) {
                     double p = __dadd_rn(base, term[b]);
                     if (p < p_min) p = p_min;
                     if (p > p_max) p = p_max;
-                    e = __dadd_rn(e, __dmul_rn(weight[b], p));
+                    prod[b] = __dmul_rn(weight[b], p);
                 }
-                e = __ddiv_rn(e, n);
-                if (e < kappa) lo = mid; else hi = mid;
+                __syncwarp();
+                int below = 0;
+                if (lane == 0) {
+                    double e = 0.0;
+#pragma unroll 8
+                    for (int b = 0; b < B; ++b) e = __dadd_rn(e, prod[b]);
+                    below = __ddiv_rn(e, n) < kappa ? 1 : 0;
+                }
+                below = __shfl_sync(0xffffffffu, below, 0);       // also orders the reads of prod before the next writes
+                if (below) lo = mid; else hi = mid;
             }
             delta = __dmul_rn(0.5, __dadd_rn(lo, hi));
         }
-        hd->delta = delta;
+        if (lane == 0) hd->delta = delta;
     }
 }
 
