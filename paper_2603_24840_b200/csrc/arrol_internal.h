@@ -90,4 +90,10 @@ int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_str
 // ARROL_ERR_UNSUPPORTED (nothing launched) when the sizes do not fit the context's buffers.
 int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index,
                                 int N, const arrol_head* head, int B, const float* q_lut, float* score, float* prob,
-                                int32_t* bin, float* q, cudaStream_t s);
+                                int32_t* bin, float* q, float* u_out /* [N][h] pre-activations, or NULL */,
+                                cudaStream_t s);
+
+// lm_head_backward.cu: C[M,N] (+)= A^T B on the tensor cores, A stored [K, M] and B stored [K, N] row-major bf16
+// (rows lda / ldb elements apart, multiples of 8), C fp32 with rows ldc apart.  Rows past K read as zero.
+int arrol_internal_gemm_tn(arrol_ctx* ctx, const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K,
+                           float* C, int64_t ldc, int accumulate, cudaStream_t s);

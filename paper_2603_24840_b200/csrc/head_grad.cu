@@ -12,6 +12,7 @@
 namespace {
 
 constexpr int DS_THREADS = 1024;
+constexpr int DU_RUNS = 32;          // row runs of the du kernel on the tensor-core path
 
 __device__ __forceinline__ double block_sum(double v, double* sh /* [32] */) {
 #pragma unroll
@@ -114,7 +115,8 @@ __global__ void column_sum_kernel(const float* __restrict__ partial, int chunks,
 template <typename T>
 __global__ void __launch_bounds__(256)
 mlp_du_kernel(const float* __restrict__ u, const float* __restrict__ ds, const T* __restrict__ w2, int N, int h,
-              float* __restrict__ du, float* __restrict__ dw2, float* __restrict__ db1) {
+              float* __restrict__ du, __nv_bfloat16* __restrict__ du_hi, __nv_bfloat16* __restrict__ du_lo,
+              float* __restrict__ dw2, float* __restrict__ db1, int rows_per_block) {
     __shared__ float sh_w2[8][33], sh_b1[8][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int j = blockIdx.x * 32 + tx;
@@ -122,13 +124,22 @@ mlp_du_kernel(const float* __restrict__ u, const float* __restrict__ ds, const T
     if (j < h) {
         float wj;
         if constexpr (sizeof(T) == 2) wj = __bfloat162float(w2[j]); else wj = w2[j];
-        for (int i = ty; i < N; i += 8) {
+        // blockIdx.y picks a run of rows; its sums go to row blockIdx.y of dw2 / db1 ([gridDim.y][h]), added up in
+        // index order by column_sum_kernel when there is more than one run
+        const int i_begin = blockIdx.y * rows_per_block, i_end = min(N, i_begin + rows_per_block);
+        for (int i = i_begin + ty; i < i_end; i += 8) {
             const float g = ds[i];
             const float a = u[(int64_t)i * h + j];
             const float cdf = 0.5f * (1.0f + erff(a * 0.70710678118654752440f));
             const float pdf = expf(-0.5f * a * a) * 0.39894228040143267794f;
             const float d_u = g * wj * (cdf + a * pdf);
-            du[(int64_t)i * h + j] = d_u;
+            if (du_hi) {       // du as the sum of two bf16 numbers (error 2^-17 relative): the tensor-core operand
+                const __nv_bfloat16 hi = __float2bfloat16_rn(d_u);
+                du_hi[(int64_t)i * h + j] = hi;
+                du_lo[(int64_t)i * h + j] = __float2bfloat16_rn(d_u - __bfloat162float(hi));
+            } else {
+                du[(int64_t)i * h + j] = d_u;
+            }
             a_w2 = fmaf(g, a * cdf, a_w2);
             a_b1 += d_u;
         }
@@ -139,8 +150,8 @@ mlp_du_kernel(const float* __restrict__ u, const float* __restrict__ ds, const T
     if (ty == 0 && j < h) {
         float s1 = 0.f, s2 = 0.f;
         for (int r = 0; r < 8; ++r) { s1 += sh_w2[r][tx]; s2 += sh_b1[r][tx]; }
-        dw2[j] = s1;
-        db1[j] = s2;
+        dw2[(int64_t)blockIdx.y * h + j] = s1;
+        db1[(int64_t)blockIdx.y * h + j] = s2;
     }
 }
 
@@ -205,6 +216,7 @@ mlp_dw1_kernel(const float* __restrict__ du, const T* __restrict__ hidden, int64
 
 struct GradLayout {
     size_t tmp3, ds, u, du, partial, total;   // byte offsets
+    size_t du_plane;                          // bytes of one bf16 plane of du (hi at du, lo at du + du_plane)
 };
 GradLayout grad_layout(int N, int d, int h) {
     GradLayout L;
@@ -213,10 +225,14 @@ GradLayout grad_layout(int N, int d, int h) {
     L.tmp3 = o; o = up(o + sizeof(float) * 3 * (size_t)N);
     L.ds = o; o = up(o + sizeof(float) * (size_t)N);
     L.u = o; o = up(o + sizeof(float) * (size_t)N * (size_t)(h > 0 ? h : 0));
-    L.du = o; o = up(o + sizeof(float) * (size_t)N * (size_t)(h > 0 ? h : 0));
+    const size_t plane = up(sizeof(uint16_t) * (size_t)N * (size_t)(h > 0 ? h : 0));   // one bf16 plane of du
+    L.du = o; o = up(o + (sizeof(float) * (size_t)N * (size_t)(h > 0 ? h : 0) > 2 * plane
+                              ? sizeof(float) * (size_t)N * (size_t)(h > 0 ? h : 0) : 2 * plane));
+    L.du_plane = plane;
     const size_t chunks = ((size_t)N + LIN_ROWS - 1) / LIN_ROWS;
     const size_t tiles = (size_t)((h > 0 ? h : 0) + ARROL_MLP_TH - 1) / ARROL_MLP_TH;
-    const size_t part = h > 0 ? tiles * (size_t)N : chunks * (size_t)d;
+    size_t part = h > 0 ? tiles * (size_t)N : chunks * (size_t)d;
+    if (h > 0 && part < 2 * (size_t)DU_RUNS * (size_t)h) part = 2 * (size_t)DU_RUNS * (size_t)h;   // dw2 / db1 per row run
     L.partial = o; o = up(o + sizeof(float) * part);
     L.total = o;
     return L;
@@ -244,12 +260,45 @@ int run_head_grad(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const 
     } else {
         float* u = reinterpret_cast<float*>(ws + L.u);
         float* du = reinterpret_cast<float*>(ws + L.du);
+        if constexpr (sizeof(T) == 2) {
+            // bf16 head: both contractions on the tensor cores.  Forward with the pre-activations kept, du split into
+            // two bf16 planes, dW1 = du_hi^T X + du_lo^T X with X the packed rows (or the rows in place).
+            if (h % 8 == 0) {
+                float* tmp = reinterpret_cast<float*>(ws + L.tmp3);
+                const int rc = arrol_internal_score_mlp_tc(ctx, hidden, row_stride, row_index, N, head, 0, nullptr, tmp,
+                                                           tmp + N, nullptr, tmp + 2 * (size_t)N, u, s);
+                if (rc == ARROL_OK) {
+                    __nv_bfloat16* du_hi = reinterpret_cast<__nv_bfloat16*>(ws + L.du);
+                    __nv_bfloat16* du_lo = reinterpret_cast<__nv_bfloat16*>(ws + L.du + L.du_plane);
+                    head_ds_kernel<T><<<1, DS_THREADS, 0, s>>>(tmp, nullptr, 0, nullptr, N, rewards, mask, ds, loss, db2);
+                    // the tile partials are consumed by now: the region holds the per-run sums of dw2 and db1
+                    const int rows_per = ((N + DU_RUNS - 1) / DU_RUNS + 7) / 8 * 8;
+                    const int runs = (N + rows_per - 1) / rows_per;
+                    float* dw2_runs = partial;
+                    float* db1_runs = partial + (size_t)DU_RUNS * h;
+                    mlp_du_kernel<T><<<dim3((h + 31) / 32, runs), 256, 0, s>>>(u, ds, static_cast<const T*>(head->w2), N, h,
+                                                                               nullptr, du_hi, du_lo, dw2_runs, db1_runs,
+                                                                               rows_per);
+                    column_sum_kernel<<<(h + 255) / 256, 256, 0, s>>>(dw2_runs, runs, h, dw2);
+                    column_sum_kernel<<<(h + 255) / 256, 256, 0, s>>>(db1_runs, runs, h, db1);
+                    ctx->launches += 4;
+                    ARROL_CUDA_OK(cudaGetLastError());
+                    const void* x = row_index ? ctx->d_pack : hidden;
+                    const int64_t ldx = row_index ? d : row_stride;
+                    int rg = arrol_internal_gemm_tn(ctx, du_hi, h, x, ldx, h, d, N, dW1, d, 0, s);
+                    if (rg == ARROL_OK) rg = arrol_internal_gemm_tn(ctx, du_lo, h, x, ldx, h, d, N, dW1, d, 1, s);
+                    return rg;
+                }
+                if (rc != ARROL_ERR_UNSUPPORTED) return rc;
+            }
+        }
         const int rc = arrol_internal_mlp_tiles(ctx, hidden, row_stride, row_index, N, head, partial, u, s);
         if (rc != ARROL_OK) return rc;
         const int h_tiles = (h + ARROL_MLP_TH - 1) / ARROL_MLP_TH;
         head_ds_kernel<T><<<1, DS_THREADS, 0, s>>>(nullptr, partial, h_tiles, static_cast<const T*>(head->b2), N,
                                                    rewards, mask, ds, loss, db2);
-        mlp_du_kernel<T><<<(h + 31) / 32, 256, 0, s>>>(u, ds, static_cast<const T*>(head->w2), N, h, du, dw2, db1);
+        mlp_du_kernel<T><<<(h + 31) / 32, 256, 0, s>>>(u, ds, static_cast<const T*>(head->w2), N, h, du, nullptr,
+                                                       nullptr, dw2, db1, N);
         dim3 grid((d + GT - 1) / GT, (h + GT - 1) / GT);
         mlp_dw1_kernel<T><<<grid, 128, 0, s>>>(du, hid, row_stride, row_index, N, d, h, dW1);
         ctx->launches += 3;

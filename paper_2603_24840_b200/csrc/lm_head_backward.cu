@@ -478,6 +478,27 @@ BackwardLayout backward_layout(int d, int V) {
 
 }  // namespace
 
+int arrol_internal_gemm_tn(arrol_ctx* ctx, const void* A, int64_t lda, const void* B, int64_t ldb, int M, int N, int K,
+                           float* C, int64_t ldc, int accumulate, cudaStream_t s) {
+    if (M <= 0 || N <= 0 || K <= 0 || lda % 8 != 0 || ldb % 8 != 0) return ARROL_ERR_UNSUPPORTED;
+    ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    CUtensorMap map_a, map_b;
+    bool a3 = M % 64 == 0, b3 = N % 64 == 0;
+    if (a3 && make_map_mn3d(ctx, &map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM / 64) != ARROL_OK) a3 = false;
+    if (b3 && make_map_mn3d(ctx, &map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, BN / 64) != ARROL_OK) b3 = false;
+    if (!a3 && make_map_ld(ctx, &map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+    if (!b3 && make_map_ld(ctx, &map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, BK) != ARROL_OK) return ARROL_ERR_CUDA;
+    GemmParams g;
+    g.M = M; g.N = N; g.K = K; g.C = C; g.ldc = ldc; g.accumulate = accumulate; g.k_is_tokens = 0;
+    g.a3d = a3; g.b3d = b3; g.d_T = nullptr; g.T_max = 1; g.t0 = 0; g.d_status = ctx->d_status;
+    const int64_t items = (int64_t)((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    gemm_kernel<true, true><<<(unsigned)(items < ctx->sm_count ? items : ctx->sm_count), NUM_THREADS, SMEM_BYTES, s>>>(
+        map_a, map_b, map_b, g);
+    ctx->launches += 1;
+    ARROL_CUDA_OK(cudaGetLastError());
+    return ARROL_OK;
+}
+
 extern "C" size_t arrol_lm_head_backward_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
     if (!ctx || T_max <= 0 || d <= 0 || V <= 0) return 0;
     return backward_layout(d, V).total;

@@ -293,7 +293,7 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
             // bf16 head: the first layer is a dense contraction, so the whole head runs on the tensor-core path
             // when the context's buffers hold the problem
             const int rc = arrol_internal_score_mlp_tc(ctx, hidden, row_stride, row_index, N, head, B, q_lut, score,
-                                                       prob, bin, q, s);
+                                                       prob, bin, q, nullptr, s);
             if (rc != ARROL_ERR_UNSUPPORTED) return rc;
         }
         const int h_tiles = (head->h + TH - 1) / TH;

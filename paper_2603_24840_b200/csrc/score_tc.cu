@@ -63,6 +63,7 @@ struct ScoreTcParams {
     const __nv_bfloat16* w2;           // [h]
     const __nv_bfloat16* b2;           // [1] or NULL
     float* partial;                    // [h_tiles][N]
+    float* u_out;                      // [N][h] pre-activations (bias included) for the head training step, or NULL
     uint32_t* counters;                // [row tiles], zero between calls
     int B;
     const float* q_lut;
@@ -199,8 +200,16 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 #pragma unroll
                 for (int jj = 0; jj < 32; ++jj) {
                     const float u = v[jj] + b1_s[piece * 32 + jj];
+                    v[jj] = u;
                     const float g = 0.5f * u * (1.0f + erff(u * 0.70710678118654752440f));
                     part = fmaf(w2_s[piece * 32 + jj], g, part);
+                }
+                if (p.u_out && m < p.N) {
+                    float* urow = p.u_out + (int64_t)m * p.h + j0 + piece * 32;
+#pragma unroll
+                    for (int jj = 0; jj < 32; jj += 4)      // h % 4 == 0: a float4 never straddles the edge
+                        if (j0 + piece * 32 + jj < p.h)
+                            *reinterpret_cast<float4*>(urow + jj) = make_float4(v[jj], v[jj + 1], v[jj + 2], v[jj + 3]);
                 }
             }
         }
@@ -241,7 +250,7 @@ score_mlp_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 // do not fit the context's buffers; the caller then takes the SIMT path.
 int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index,
                                 int N, const arrol_head* head, int B, const float* q_lut, float* score, float* prob,
-                                int32_t* bin, float* q, cudaStream_t s) {
+                                int32_t* bin, float* q, float* u_out, cudaStream_t s) {
     const int d = head->d, h = head->h;
     const int m_tiles = (N + SBM - 1) / SBM, h_tiles = (h + SBN - 1) / SBN;
     if ((size_t)N * (size_t)h_tiles > ARROL_SCRATCH_FLOATS || m_tiles > ARROL_TILE_COUNTERS)
@@ -271,6 +280,7 @@ int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_
     p.w2 = static_cast<const __nv_bfloat16*>(head->w2);
     p.b2 = static_cast<const __nv_bfloat16*>(head->b2);
     p.partial = ctx->d_scratch;
+    p.u_out = u_out;
     p.counters = ctx->d_tile_counters;
     p.B = B;
     p.q_lut = q_lut;
