@@ -196,10 +196,15 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                     float v[32];
                     tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
                     if constexpr (CONF) {                   // sum of the valid logits of the piece (before masking)
-                        float ps = 0.f;
+                        float ps[4] = {0.f, 0.f, 0.f, 0.f};           // four chains; only the last piece needs the mask
+                        if (pc0 + 32 <= p.V) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) ps += (pc0 + j < p.V) ? v[j] : 0.f;
-                        sumz += ps;
+                            for (int j = 0; j < 32; ++j) ps[j & 3] += v[j];
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) ps[j & 3] += (pc0 + j < p.V) ? v[j] : 0.f;
+                        }
+                        sumz += (ps[0] + ps[1]) + (ps[2] + ps[3]);
                     }
                     if (pc0 + 32 > p.V) {
 #pragma unroll
