@@ -16,6 +16,8 @@ struct arrol_ctx {
     float* d_scratch;          // MLP-head partial sums: [ARROL_SCRATCH_FLOATS]
     void* d_pack;              // MLP head on the tensor cores: the scored rows packed as bf16 [N][d], ARROL_PACK_BYTES
     uint32_t* d_tile_counters; // MLP head on the tensor cores: finished blocks per row tile, zero between calls
+    bool score_tc_smem_set;    // the scoring kernel's dynamic shared-memory limit has been raised on this device
+    bool gather_bulk_smem_set; // likewise for the bulk-copy gather kernel
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
     unsigned long long launches;   // kernels launched through this context (host-side count)
     cudaStream_t copy_stream;      // second stream of the host-buffer step: uploads overlap the log-prob kernel
@@ -61,8 +63,18 @@ struct ArrolDeviceGuard {
 // run back to back on one stream and last a few microseconds each: a kernel launched with arrol_launch_pdl may
 // start while its predecessor is still running, sets up (shared memory, barriers, tensor-map prefetch) and then
 // blocks in pdl_wait() until the predecessor has completed and its writes are visible.  Every such kernel calls
-// pdl_launch_dependents() at its top and touches global memory only after pdl_wait().
+// pdl_launch_dependents() at its top and touches global memory only after pdl_wait(), through pointers passed
+// through pdl_acquire().
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// A kernel that may start before its predecessor has finished must not load the predecessor's results early.  The
+// compiler is free to hoist loads through `const __restrict__` pointers (read-only data by contract) above the wait,
+// so every pointer to data an earlier kernel may have written is passed through this after pdl_wait(): the loads
+// then depend on a value produced after the wait.
+template <typename T>
+__device__ __forceinline__ T* pdl_acquire(T* p) {
+    asm volatile("" : "+l"(p) :: "memory");
+    return p;
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
@@ -92,6 +104,12 @@ int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_
                                 int N, const arrol_head* head, int B, const float* q_lut, float* score, float* prob,
                                 int32_t* bin, float* q, float* u_out /* [N][h] pre-activations, or NULL */,
                                 cudaStream_t s);
+
+// gather_bulk.cu: the survivors' rows moved by bulk copies through shared memory.  ARROL_ERR_UNSUPPORTED (nothing
+// launched) when a row does not fit a 32 KB stage.
+int arrol_internal_gather_rows_bulk(arrol_ctx* ctx, const int64_t* d_num, const int64_t* cu_seqlens,
+                                    const int32_t* survivor_idx, const int64_t* src_tok_off, const void* src_rows,
+                                    int64_t row_bytes, int64_t capacity, void* dst_rows, cudaStream_t s);
 
 // lm_head_backward.cu: C[M,N] (+)= A^T B on the tensor cores, A stored [K, M] and B stored [K, N] row-major bf16
 // (rows lda / ldb elements apart, multiples of 8), C fp32 with rows ldc apart.  Rows past K read as zero.

@@ -4,10 +4,11 @@
 // Kernel 1 (one block): stable partition by a block-wide prefix sum over (kept flag, kept length):
 //   survivor_idx, cu_seqlens, {S, T}, and per-survivor advantages (fp64 statistics over the kept rollouts of
 //   the group, in index order, rounded once to fp32).
-// Kernel 2 (one wave of persistent blocks): moves the survivors' rows.  Each block owns a contiguous run of
-//   destination tiles (~32 KB of rows each); one thread per row finds its survivor (binary search once per
-//   block, then a forward walk in cu_seqlens) and writes the per-token outputs (token id, survivor ordinal,
-//   advantage); the block then streams the tile's payload with 16-byte loads/stores, eight in flight per thread.
+// Kernel 2: the per-token outputs (token id, survivor ordinal, advantage), one block per survivor, and, when there is
+//   a hidden-row plane, the rows themselves by bulk copies through shared memory (gather_bulk.cu).  Rows too large
+//   for a bulk stage take gather_kernel below: one wave of persistent blocks, each owning a contiguous run of
+//   destination tiles; one thread per row finds its survivor (binary search once per block, then a forward walk in
+//   cu_seqlens), then the block streams the tile's payload with 16-byte loads/stores, eight in flight per thread.
 //   T is read from device memory, so there is no host synchronisation between the kernels.
 #include "arrol_internal.h"
 
@@ -37,6 +38,7 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     const bool shared_stats = G >= 4;
     pdl_launch_dependents();
     pdl_wait();
+    keep = pdl_acquire(keep); lengths = pdl_acquire(lengths); rewards = pdl_acquire(rewards);
     if (threadIdx.x == 0) { carry_cnt = 0; carry_tok = 0; cu_seqlens[0] = 0; }
     __syncthreads();
 
@@ -223,6 +225,9 @@ gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_
     __shared__ int s_first[2];               // survivor of the first row of the current / next tile
     pdl_launch_dependents();
     pdl_wait();
+    d_num = pdl_acquire(d_num); cu_seqlens = pdl_acquire(cu_seqlens); survivor_idx = pdl_acquire(survivor_idx);
+    src_tok_off = pdl_acquire(src_tok_off); src_tokens = pdl_acquire(src_tokens); src_rows = pdl_acquire(src_rows);
+    adv = pdl_acquire(adv);
     const int S = (int)d_num[0];
     const int64_t T = d_num[1];
     if (T > capacity || S <= 0 || T <= 0) return;      // capacity overflow was recorded by the scan kernel
@@ -288,6 +293,8 @@ gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restric
                      int32_t* __restrict__ dst_tokens, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
     pdl_launch_dependents();
     pdl_wait();
+    d_num = pdl_acquire(d_num); cu_seqlens = pdl_acquire(cu_seqlens); survivor_idx = pdl_acquire(survivor_idx);
+    src_tok_off = pdl_acquire(src_tok_off); src_tokens = pdl_acquire(src_tokens); adv = pdl_acquire(adv);
     const int S = (int)d_num[0];
     if (d_num[1] > capacity) return;                       // capacity overflow was recorded by the scan kernel
     for (int s = blockIdx.x; s < S; s += gridDim.x) {
@@ -346,7 +353,16 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
 
     const int vec_per_row = src_rows ? row_bytes / 16 : 0;
-    if (vec_per_row == 0) {
+    // Rows that fit a 32 KB stage go through the bulk-copy kernel; the per-token outputs then come from the
+    // survivor-major kernel.  Larger rows take the load/store kernel, which writes both.
+    const bool bulk_rows = vec_per_row > 0 && row_bytes <= 32 * 1024;
+    if (vec_per_row == 0 || bulk_rows) {
+        if (bulk_rows) {
+            const int rc = arrol_internal_gather_rows_bulk(ctx, d_num, cu_seqlens, survivor_idx, src_tok_off, src_rows,
+                                                           row_bytes, dst_capacity_tokens, dst_rows, s);
+            if (rc != ARROL_OK) return rc;
+            if (!dst_tokens && !tok_adv && !tok_seq) return ARROL_OK;
+        }
         int64_t blocks = N < (int64_t)ctx->sm_count * 16 ? N : (int64_t)ctx->sm_count * 16;
         ARROL_CUDA_OK(arrol_launch_pdl(gather_tokens_kernel, dim3((unsigned)blocks), dim3(TOKENS_THREADS), 0, s, d_num,
                                        cu_seqlens, survivor_idx, src_tok_off, src_tokens, adv, dst_capacity_tokens,

@@ -44,6 +44,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->d_scratch = nullptr;
     ctx->d_pack = nullptr;
     ctx->d_tile_counters = nullptr;
+    ctx->score_tc_smem_set = false;
+    ctx->gather_bulk_smem_set = false;
     ctx->encode_tiled = nullptr;
     ctx->launches = 0;
     ctx->copy_stream = nullptr;

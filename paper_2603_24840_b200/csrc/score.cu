@@ -64,6 +64,8 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
     constexpr int VN = Vec16<T>::N;
     pdl_launch_dependents();
     pdl_wait();
+    hidden = pdl_acquire(hidden); row_index = pdl_acquire(row_index); w = pdl_acquire(w); bias = pdl_acquire(bias);
+    q_lut = pdl_acquire(q_lut);
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= N) return;

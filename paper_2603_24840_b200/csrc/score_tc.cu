@@ -39,6 +39,7 @@ pack_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t row_stride, c
                  int N, int d, __nv_bfloat16* __restrict__ out) {
     pdl_launch_dependents();
     pdl_wait();
+    hidden = pdl_acquire(hidden); row_index = pdl_acquire(row_index);
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (i >= N) return;
@@ -289,8 +290,11 @@ int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_
     p.bin = bin;
     p.q = q;
     p.d_status = ctx->d_status;
-    ARROL_CUDA_OK(cudaFuncSetAttribute(score_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)S_SMEM_BYTES));
+    if (!ctx->score_tc_smem_set) {      // once per context: this call is on the prune step's microsecond path
+        ARROL_CUDA_OK(cudaFuncSetAttribute(score_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)S_SMEM_BYTES));
+        ctx->score_tc_smem_set = true;
+    }
     dim3 grid(m_tiles, h_tiles);
     ARROL_CUDA_OK(arrol_launch_pdl(score_mlp_tc_kernel, grid, dim3(S_THREADS), S_SMEM_BYTES, s, map_x, map_w, p));
     ctx->launches += 1;

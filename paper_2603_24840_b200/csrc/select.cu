@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(128)
 select_kernel(const float* __restrict__ q, int P, int G, int K, double rho, int seg, uint8_t* __restrict__ keep) {
     pdl_launch_dependents();
     pdl_wait();
+    q = pdl_acquire(q);
     const int lane = threadIdx.x & 31;
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int groups_per_warp = 32 / seg;
