@@ -76,3 +76,43 @@ def test_prune_step_replayed_from_a_cuda_graph(name, rows):
     assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
     del graph
     pr.ctx.close()
+
+
+def test_back_to_back_steps_never_read_the_previous_steps_results():
+    """The kernels of a step start while their predecessor is still running (programmatic dependent launch) and must
+    wait before they read its results.  Two steps with different heads are issued back to back without a host
+    synchronisation; the buffers must hold exactly what the second step alone produces, in either order."""
+    w = synth.WORKLOADS["profile-mlp"]
+    pr = PruneRebatch(w, inputs=host_inputs(w), with_rows=False)
+    heads = [pr.head, dict(pr.head)]
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    heads[1]["w2"] = (pr.head["w2"].float() * (torch.rand(w.h, generator=gen, device="cuda") * 4 - 2)).to(pr.head["w2"].dtype)
+    keys = ("score", "q", "keep", "survivor_idx", "cu_seqlens", "adv", "d_num", "dst_tokens", "tok_seq")
+    refs = []
+    for hd in heads:
+        pr.head = hd
+        B.arrol_prune_step(pr.ctx, pr.prune_step_args(with_rows=False))
+        torch.cuda.synchronize()
+        refs.append(({k: getattr(pr, k).clone() for k in keys}, pr.counts()))
+    assert not torch.equal(refs[0][0]["keep"], refs[1][0]["keep"])          # the two steps really differ
+    args = []
+    for hd in heads:
+        pr.head = hd
+        args.append(pr.prune_step_args(with_rows=False))
+    for first, second in ((0, 1), (1, 0), (0, 1)):
+        for _ in range(3):
+            B.arrol_prune_step(pr.ctx, args[first])
+            B.arrol_prune_step(pr.ctx, args[second])
+        torch.cuda.synchronize()
+        want, (S, T) = refs[second]
+        assert pr.counts() == (S, T)
+        for k in ("score", "q", "keep", "d_num"):
+            assert torch.equal(getattr(pr, k), want[k]), k
+        for k in ("survivor_idx", "adv"):
+            assert torch.equal(getattr(pr, k)[:S], want[k][:S]), k
+        assert torch.equal(pr.cu_seqlens[:S + 1], want["cu_seqlens"][:S + 1])
+        for k in ("dst_tokens", "tok_seq"):
+            assert torch.equal(getattr(pr, k)[:T], want[k][:T]), k
+    assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+    pr.ctx.close()
