@@ -403,7 +403,6 @@ def run_ours(args, w):
                                  "algorithmic_bytes_per_launch": gather_bytes},
         }
         esz = pr.hidden_score.element_size()
-        props = torch.cuda.get_device_properties(local)
         if w.h == 0:
             gbs = n_score * w.d * esz / (score_ms * 1e-3) / 1e9
             out["score_roofline"] = {"kernel": "score_linear_kernel", "bound": "hbm", "rows": int(n_score),
@@ -559,7 +558,7 @@ def auto_prompt_chunks(w):
 def run_e2e(args, w, pr, B, torch, world, barrier):
     """Same step through the host-buffer entry point: every step copies the inputs from pinned host memory and
     reads the results back."""
-    N, cap, d = w.N, pr.cap, w.d
+    N, cap = w.N, pr.cap
     pin = lambda t: t.cpu().pin_memory()
     h = {
         "h_hidden": pin(pr.src_rows), "h_src_tokens": pin(pr.src_tokens), "h_lengths": pin(pr.lengths),
@@ -588,7 +587,7 @@ def run_e2e(args, w, pr, B, torch, world, barrier):
     step = B.make_host_step(scal, head, pr.q_lut, tensors)
     # bytes the call moves per step: small arrays and token ids, the N hidden rows at the detection length, then only
     # the survivors' hidden rows (uploaded straight into their packed positions); results: logp[T] + per-rollout arrays
-    S_now, T_now = pr.counts()
+    _, T_now = pr.counts()
     row_bytes = w.d * 2
     h2d = sum(h[k].numel() * h[k].element_size() for k in ("h_src_tokens", "h_lengths", "h_src_tok_off", "h_rewards"))
     h2d += (N + T_now) * row_bytes
