@@ -242,7 +242,8 @@ def _compact_case(ctx, N, G, row_bytes, seed, keep_prob=0.5, lo=0, hi=40, padded
 
 
 @pytest.mark.parametrize("N,G,row_bytes", [(32, 8, 0), (32, 8, 1024), (2048, 16, 64), (4096, 16, 0),
-                                           (5000, 8, 16), (96, 32, 4096), (48, 16, 8192 + 16)])
+                                           (5000, 8, 16), (96, 32, 4096), (48, 16, 8192 + 16),
+                                           (24, 8, 32768), (24, 8, 32768 + 64)])   # largest bulk-copy row; load/store kernel
 def test_compact_matches_oracle(ctx, N, G, row_bytes):
     _compact_case(ctx, N, G, row_bytes, seed=N + row_bytes)
     _compact_case(ctx, N, G, row_bytes, seed=N + row_bytes + 1, padded=True, ddof=1)
