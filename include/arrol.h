@@ -398,6 +398,19 @@ int arrol_score_partial_static(const void* hidden, int64_t row_stride_elems, con
 /* Number of kernels this context has launched so far (host-side count; -1 for a NULL context). */
 int64_t arrol_launch_count(arrol_ctx* ctx);
 
+/* ---- Test hook (no counterpart in the paper) --------------------------------------------------------------------
+ * Every pipeline wait inside the tensor-core kernels is bounded: when one runs out the block records
+ * ARROL_DEV_WAIT_EXPIRED, lets its copies and MMAs in flight finish, frees its tensor memory and returns, and the
+ * context stays usable.  In correct operation no wait ever runs out, so this hook lets a test exercise that path of
+ * arrol_token_logprob without a fault or a hang:
+ *   ARROL_HOOK_SPIN_LIMIT            value = tries per wait (0 restores the normal limit of 2^26)
+ *   ARROL_HOOK_MUTE_LOGPROB_PRODUCER value != 0: the kernel's producer issues no copies, so the other roles' waits
+ *                                    run out after the limit above; outputs of such a call are not written.
+ * Returns INVALID_ARG for an unknown key or a limit outside [0, 2^26]. */
+#define ARROL_HOOK_SPIN_LIMIT 1
+#define ARROL_HOOK_MUTE_LOGPROB_PRODUCER 2
+int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value);
+
 #ifdef __cplusplus
 }
 #endif

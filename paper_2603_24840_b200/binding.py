@@ -26,7 +26,7 @@ EXPORTS = [
     "arrol_calib_delta", "arrol_select_stochastic",
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
     "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
-    "arrol_prune_step", "arrol_token_logprob_splits",
+    "arrol_prune_step", "arrol_token_logprob_splits", "arrol_test_hook",
 ]
 
 
@@ -271,6 +271,16 @@ def arrol_token_logprob(ctx: Context, hidden, W_vocab, targets, T_max: int, d: i
                                               _ptr(lse), _ptr(workspace),
                                               0 if workspace is None else workspace.numel() * workspace.element_size(),
                                               _stream(stream)), "arrol_token_logprob")
+
+
+HOOK_SPIN_LIMIT, HOOK_MUTE_LOGPROB_PRODUCER = 1, 2
+
+
+def arrol_test_hook(ctx: Context, key: int, value: int):
+    """Test hook: bounds the log-prob kernel's pipeline waits / silences its producer (see include/arrol.h)."""
+    lib = load_library()
+    lib.arrol_test_hook.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
+    _check(lib.arrol_test_hook(ctx.handle, int(key), int(value)), "arrol_test_hook")
 
 
 def arrol_launch_count(ctx: Context) -> int:

@@ -18,6 +18,8 @@ struct arrol_ctx {
     uint32_t* d_tile_counters; // MLP head on the tensor cores: finished blocks per row tile, zero between calls
     bool score_tc_smem_set;    // the scoring kernel's dynamic shared-memory limit has been raised on this device
     bool gather_bulk_smem_set; // likewise for the bulk-copy gather kernel
+    uint32_t test_spin_limit;  // arrol_test_hook: tries per pipeline wait of the log-prob kernel, 0 = the normal limit
+    int test_mute_producer;    // arrol_test_hook: the log-prob kernel's producer issues no copies (its waits run out)
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
     unsigned long long launches;   // kernels launched through this context (host-side count)
     cudaStream_t copy_stream;      // second stream of the host-buffer step: uploads overlap the log-prob kernel

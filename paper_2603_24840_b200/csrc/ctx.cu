@@ -46,6 +46,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->d_tile_counters = nullptr;
     ctx->score_tc_smem_set = false;
     ctx->gather_bulk_smem_set = false;
+    ctx->test_spin_limit = 0;
+    ctx->test_mute_producer = 0;
     ctx->encode_tiled = nullptr;
     ctx->launches = 0;
     ctx->copy_stream = nullptr;
@@ -95,6 +97,21 @@ extern "C" int arrol_destroy(arrol_ctx* ctx) {
 }
 
 extern "C" int64_t arrol_launch_count(arrol_ctx* ctx) { return ctx ? (int64_t)ctx->launches : -1; }
+
+extern "C" int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value) {
+    if (!ctx) return ARROL_ERR_INVALID_ARG;
+    switch (key) {
+        case ARROL_HOOK_SPIN_LIMIT:
+            if (value < 0 || value > (int64_t)1 << 26) return ARROL_ERR_INVALID_ARG;
+            ctx->test_spin_limit = (uint32_t)value;
+            return ARROL_OK;
+        case ARROL_HOOK_MUTE_LOGPROB_PRODUCER:
+            ctx->test_mute_producer = value != 0;
+            return ARROL_OK;
+        default:
+            return ARROL_ERR_INVALID_ARG;
+    }
+}
 
 extern "C" int arrol_poll_status(arrol_ctx* ctx, void* stream, uint32_t* dev_status_bits) {
     if (!ctx) return ARROL_ERR_INVALID_ARG;

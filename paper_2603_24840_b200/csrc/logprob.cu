@@ -48,6 +48,8 @@ struct LogprobParams {
     float* conf;           // token confidence H_t = -sum_v log P_t(v) = V lse - sum_v z_v, or NULL
     float inv_temp;
     PartialLse* partial;   // [splits][T_max] when splits > 1
+    uint32_t spin_limit;   // tries per pipeline wait
+    int mute_producer;     // test hook: the producer issues no copies
     uint32_t* d_status;
 };
 
@@ -102,13 +104,13 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            for (int64_t item = blockIdx.x; item < items && ok && !p.mute_producer; item += gridDim.x) {
                 const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
                 const int c0 = split * p.chunks_per_split;
                 const int c1 = min(c0 + p.chunks_per_split, total_chunks);
                 for (int c = c0; c < c1 && ok; ++c) {
                     for (int ks = 0; ks < k_steps; ++ks) {
-                        if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
                         mbar_expect_tx(&full[stage], STAGE_BYTES);
                         tma_load_2d(stage_a + (size_t)stage * A_STAGE_BYTES, &map_h, ks * BK, m_tile * BM, &full[stage]);
                         tma_load_2d(stage_b + (size_t)stage * B_STAGE_BYTES, &map_w, ks * BK, c * BN, &full[stage]);
@@ -124,7 +126,7 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 uint32_t s = stage, ph = phase;
                 for (uint32_t i = 0; i < pending; ++i) {
                     if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
-                    for (uint32_t it = 0; it < SPIN_LIMIT; ++it)
+                    for (uint32_t it = 0; it < p.spin_limit; ++it)
                         if (mbar_try_wait(&full[s], ph)) break;
                 }
             }
@@ -141,11 +143,11 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 const int c0 = split * p.chunks_per_split;
                 const int c1 = min(c0 + p.chunks_per_split, total_chunks);
                 for (int c = c0; c < c1 && ok; ++c) {
-                    if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(&acc_empty[acc], acc_phase ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * BN;
                     for (int ks = 0; ks < k_steps; ++ks) {
-                        if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(&full[stage], phase, abort_flag, p.spin_limit)) { ok = false; break; }
                         tcgen05_fence_after();
                         const uint64_t a_desc = make_smem_desc(smem_u32(stage_a + (size_t)stage * A_STAGE_BYTES));
                         const uint64_t b_desc = make_smem_desc(smem_u32(stage_b + (size_t)stage * B_STAGE_BYTES));
@@ -165,7 +167,7 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
             if (!ok) {
                 // Gave up: wait (bounded) until the MMAs already issued have finished with shared and tensor memory.
                 tcgen05_commit(drain);
-                for (uint32_t it = 0; it < SPIN_LIMIT; ++it)
+                for (uint32_t it = 0; it < p.spin_limit; ++it)
                     if (mbar_try_wait(drain, 0u)) break;
             }
         }
@@ -184,7 +186,7 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
             const int y = (t < T) ? p.targets[t] : -1;
             float m2 = -INFINITY, l = 0.f, zy2 = -INFINITY, sumz = 0.f;
             for (int c = c0; c < c1 && ok; ++c) {
-                ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag);
+                ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.spin_limit);
                 ok = __all_sync(0xffffffffu, ok) != 0;     // keep the warp converged for the aligned tensor-memory loads
                 if (!ok) break;
                 tcgen05_fence_after();
@@ -371,6 +373,8 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     p.inv_temp = inv_temperature;
     p.partial = static_cast<PartialLse*>(workspace);
     p.d_status = ctx->d_status;
+    p.spin_limit = ctx->test_spin_limit ? ctx->test_spin_limit : SPIN_LIMIT;
+    p.mute_producer = ctx->test_mute_producer;
 
     ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)SMEM_BYTES));
