@@ -176,6 +176,14 @@ def run_reference(args, w):
     rank, world, _ = dist_env()
     if rank != 0:
         return
+    if world > 1:
+        # torchrun exports OMP_NUM_THREADS=1 to every rank; the other ranks have exited, so rank 0 times the oracle on
+        # all host cores, as the single-process run does
+        try:
+            import ctypes
+            ctypes.CDLL("libgomp.so.1").omp_set_num_threads(len(os.sched_getaffinity(0)))
+        except OSError:
+            pass
     vals = []
     budget = max(2.0, min(30.0, 120.0 / max(1, args.steps + args.warmup)))
     sample = ""
