@@ -103,3 +103,45 @@ def test_qwen3_4b_shaped():
 
 def test_qwen3_8b_dapo_shaped_one_prompt_chunk():
     _fullsize("qwen3-8b-dapo", 16, prompt_chunks=4)
+
+
+def test_llama_3_2_1b_shaped_update_leg():
+    """lm_head backward at the benchmark's size and launch configuration (all 35 token chunks of the step's survivors).
+    The gradient w.r.t. the log-probs is non-zero on a sample of tokens only (first and last rows, both sides of
+    chunk and tile edges, the last partial chunk, random ones), so the oracle can produce the exact dH rows of the
+    sample and the whole of dW = sum over the sample; every other dH row must be exactly zero."""
+    from oracle import update as ou
+    from paper_2603_24840_b200 import update as U
+    w = synth.WORKLOADS["llama-3.2-1b"]
+    pr = PruneRebatch(w, inputs=host_inputs(w))
+    pr.step()
+    torch.cuda.synchronize()
+    S, T = pr.counts()
+    g = np.random.default_rng(11)
+    chunk = 9472
+    edges = [0, 1, 127, 128, chunk - 1, chunk, chunk + 1, 5 * chunk - 1, 5 * chunk, (T // chunk) * chunk, T - 129, T - 2, T - 1]
+    sample = np.unique(np.concatenate([np.array(edges), g.integers(0, T, size=35)])).astype(np.int64)
+    grad_s = g.normal(size=sample.size).astype(np.float32)
+    grad = torch.zeros(pr.cap, device=pr.dev)
+    grad[torch.from_numpy(sample).to(pr.dev)] = torch.from_numpy(grad_s).to(pr.dev)
+    dH = torch.full((pr.cap, w.d), 9.0, device=pr.dev)
+    dW = torch.full((w.V, w.d), 9.0, device=pr.dev)
+    ws = torch.empty(U.arrol_lm_head_backward_workspace(pr.ctx, pr.cap, w.d, w.V), dtype=torch.uint8, device=pr.dev)
+    U.arrol_lm_head_backward(pr.ctx, pr.dst_rows, pr.W_vocab, pr.dst_tokens, grad, pr.lse, pr.cap, w.d, w.V, dH, dW, ws,
+                             d_T=pr.d_num[1:])
+    torch.cuda.synchronize()
+    assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+
+    idx = torch.from_numpy(sample).to(pr.dev)
+    H_s = pr.dst_rows[idx].cpu()
+    y_s = pr.dst_tokens[idx].cpu().numpy()
+    dH_ref, dW_ref = ou.lm_head_backward(synth.as_oracle_array(H_s), synth.as_oracle_array(pr.W_vocab.cpu()), y_s,
+                                         grad_s.astype(np.float64))
+    dH_s = dH[idx].cpu().numpy().astype(np.float64)
+    for got, ref in ((dH_s, dH_ref), (dW.cpu().numpy().astype(np.float64), dW_ref)):
+        assert np.abs(got - ref).max() <= 1e-2 * np.abs(ref).max()
+        assert np.linalg.norm(got - ref) <= 5e-3 * np.linalg.norm(ref)
+    rest = torch.ones(T, dtype=torch.bool, device=pr.dev)
+    rest[idx] = False
+    assert float(dH[:T][rest].abs().max()) == 0.0             # rows without a gradient are exactly zero
+    pr.ctx.close()
