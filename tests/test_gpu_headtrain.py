@@ -65,3 +65,30 @@ def test_head_grad_empty_inputs():
     torch.cuda.synchronize()
     assert loss.item() == 0.0 and torch.all(grads["W1"] == 0)
     ctx.close()
+
+
+def test_head_grad_rows_in_place_on_the_tensor_core_path():
+    """bf16 MLP head without a row index: the contractions read the rows where they are (no packing)."""
+    ctx = B.Context(0)
+    g = np.random.default_rng(21)
+    N, d, h = 200, 512, 128
+    x = torch.from_numpy(g.normal(size=(N, d)).astype(np.float32)).to(torch.bfloat16)
+    mk = lambda *s: torch.from_numpy(g.normal(0, 0.05, size=s).astype(np.float32)).to(torch.bfloat16)
+    head = {"W1": mk(h, d), "b1": mk(h), "w2": mk(h) * 4, "b2": mk(1)}
+    rew = (g.random(N) < 0.4).astype(np.float32)
+    oa = synth.as_oracle_array
+    loss_ref, gref = oh.head_bce_grad(oa(x), rew > 0.5, oa(head["W1"]), oa(head["b1"]), oa(head["w2"]), oa(head["b2"]), h=h)
+    dhead = {k: v.cuda() for k, v in head.items()}
+    dhead["h"] = h
+    grads = {"W1": torch.full((h, d), 5.0, device="cuda"), "b1": torch.full((h,), 5.0, device="cuda"),
+             "w2": torch.full((h,), 5.0, device="cuda"), "b2": torch.full((1,), 5.0, device="cuda")}
+    loss = torch.zeros(1, dtype=torch.float64, device="cuda")
+    ws = torch.empty(HT.arrol_head_grad_workspace(ctx, N, d, h), dtype=torch.uint8, device="cuda")
+    HT.arrol_head_grad(ctx, x.cuda(), dhead, N, torch.from_numpy(rew).cuda(), grads, loss, ws)
+    torch.cuda.synchronize()
+    assert abs(loss.item() - loss_ref) <= 1e-5 * max(1.0, abs(loss_ref))
+    for k, ref in gref.items():
+        got = grads[k].cpu().numpy().reshape(ref.shape).astype(np.float64)
+        assert np.abs(got - ref).max() <= 2e-4 * max(np.abs(ref).max(), 1e-6), k
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
+    ctx.close()
