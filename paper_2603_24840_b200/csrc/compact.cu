@@ -26,8 +26,6 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
                 int64_t* __restrict__ d_num, uint32_t* __restrict__ d_status) {
     __shared__ int32_t warp_cnt[32];
     __shared__ int64_t warp_tok[32];
-    __shared__ int32_t carry_cnt;
-    __shared__ int64_t carry_tok;
     // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them)
     __shared__ double g_mean[SCAN_GROUPS], g_den[SCAN_GROUPS];     // mean, 1 / (std + eps)
     // the pass's keep flags and rewards, staged once so that the statistics and the advantages read shared memory
@@ -39,8 +37,9 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     pdl_launch_dependents();
     pdl_wait();
     keep = pdl_acquire(keep); lengths = pdl_acquire(lengths); rewards = pdl_acquire(rewards);
-    if (threadIdx.x == 0) { carry_cnt = 0; carry_tok = 0; cu_seqlens[0] = 0; }
-    __syncthreads();
+    if (threadIdx.x == 0) cu_seqlens[0] = 0;
+    int32_t carry_c = 0;             // survivors / tokens of the passes so far (the same in every thread)
+    int64_t carry_t = 0;
 
     // statistics over the kept rollouts of a group (Section 3, on survivors): sums in index order, fp64
     constexpr int PASS = SCAN_THREADS * SCAN_ITEMS;
@@ -146,21 +145,21 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
         }
         if (lane == 31) { warp_cnt[wid] = c; warp_tok[wid] = t; }
         __syncthreads();
-        if (wid == 0) {
-            int32_t wc = warp_cnt[lane];
-            int64_t wt = warp_tok[lane];
+        // every warp scans the 32 warp totals itself (no second barrier, no single-warp phase)
+        int32_t wc = warp_cnt[lane];
+        int64_t wt = warp_tok[lane];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int32_t oc = __shfl_up_sync(0xffffffffu, wc, o);
-                const int64_t ot = __shfl_up_sync(0xffffffffu, wt, o);
-                if (lane >= o) { wc += oc; wt += ot; }
-            }
-            warp_cnt[lane] = wc;   // inclusive over warps
-            warp_tok[lane] = wt;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t oc = __shfl_up_sync(0xffffffffu, wc, o);
+            const int64_t ot = __shfl_up_sync(0xffffffffu, wt, o);
+            if (lane >= o) { wc += oc; wt += ot; }
         }
-        __syncthreads();
-        int32_t pos = carry_cnt + (wid ? warp_cnt[wid - 1] : 0) + (c - own_c);   // survivors before this thread's items
-        int64_t tok = carry_tok + (wid ? warp_tok[wid - 1] : 0) + (t - own_t);
+        const int32_t pass_cnt = __shfl_sync(0xffffffffu, wc, 31);          // totals of the pass
+        const int64_t pass_tok = __shfl_sync(0xffffffffu, wt, 31);
+        const int32_t before_c = __shfl_sync(0xffffffffu, wc, wid ? wid - 1 : 0);
+        const int64_t before_t = __shfl_sync(0xffffffffu, wt, wid ? wid - 1 : 0);
+        int32_t pos = carry_c + (wid ? before_c : 0) + (c - own_c);   // survivors before this thread's items
+        int64_t tok = carry_t + (wid ? before_t : 0) + (t - own_t);
 #pragma unroll
         for (int u = 0; u < SCAN_ITEMS; ++u) {
             if (!kept[u]) continue;
@@ -175,14 +174,14 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
             adv[pos] = (float)a;
             ++pos;
         }
-        __syncthreads();
-        if (threadIdx.x == 0) { carry_cnt += warp_cnt[31]; carry_tok += warp_tok[31]; }
-        __syncthreads();
+        carry_c += pass_cnt;
+        carry_t += pass_tok;
+        __syncthreads();                 // the staging arrays and warp totals are rewritten by the next pass
     }
     if (threadIdx.x == 0) {
-        d_num[0] = carry_cnt;
-        d_num[1] = carry_tok;
-        if (carry_tok > capacity) atomicOr(d_status, ARROL_DEV_CAPACITY);
+        d_num[0] = carry_c;
+        d_num[1] = carry_t;
+        if (carry_t > capacity) atomicOr(d_status, ARROL_DEV_CAPACITY);
     }
 }
 
