@@ -28,11 +28,11 @@ constexpr int TMEM_COLS = 512;
 constexpr int EPI_WARPS = 8;            // two warps per tensor-memory lane quarter, each takes half of the columns
 constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int EPI_PIECES = BN / 32 / (EPI_WARPS / 4);   // 32-column pieces per epilogue warp and accumulator
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
-// dz_kernel: one 32-row x 128-byte staging tile per epilogue warp behind the barrier block (1 KB), 1024-byte aligned
-constexpr int DZ_STAGE_TILE = 32 * 128;
-constexpr size_t DZ_STAGE_OFFSET = (size_t)STAGES * STAGE_BYTES + 1024;
-constexpr size_t DZ_SMEM_BYTES = DZ_STAGE_OFFSET + (size_t)EPI_WARPS * DZ_STAGE_TILE + 1024;
+// every kernel: one 32-row x 128-byte staging tile per epilogue warp behind the barrier block (1 KB), 1024-byte
+// aligned, from which the results leave as TMA tile stores / reductions
+constexpr int EPI_STAGE_TILE = 32 * 128;
+constexpr size_t EPI_STAGE_OFFSET = (size_t)STAGES * STAGE_BYTES + 1024;
+constexpr size_t SMEM_BYTES = EPI_STAGE_OFFSET + (size_t)EPI_WARPS * EPI_STAGE_TILE + 1024;
 constexpr int TC = 74 * BM;      // tokens per chunk: 74 token tiles, so that TC/128 x d/256 tiles fill 148 SMs evenly
 
 struct PipeSmem {
@@ -216,7 +216,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
           const __grid_constant__ CUtensorMap map_dz, const DzParams p) {
     extern __shared__ uint8_t smem_raw[];
     const PipeSmem ps = carve_smem(smem_raw);
-    uint8_t* dz_stage = ps.stage_a + DZ_STAGE_OFFSET;
+    uint8_t* dz_stage = ps.stage_a + EPI_STAGE_OFFSET;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t T = live_tokens(p.d_T, p.T_max);
     if (p.t0 >= T) return;                                  // chunk past the live tokens (uniform for the grid)
@@ -288,7 +288,7 @@ dz_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUt
             // swizzle) are staged and written by one TMA tile store, i.e. in whole 128-byte lines; columns past V are
             // clipped by the copy.  (16-byte stores straight from the registers touch 32 lines per instruction and
             // cost the kernel 14 %.)
-            uint8_t* stg = dz_stage + (size_t)(warp - 2) * DZ_STAGE_TILE;
+            uint8_t* stg = dz_stage + (size_t)(warp - 2) * EPI_STAGE_TILE;
             const int row0 = m_tile * BM + quarter * 32;
             for (int c = c0; c < c1 && ok; ++c) {
                 ok = mbar_wait(&ps.acc_full[acc], acc_phase, ps.abort_flag);
@@ -372,9 +372,11 @@ struct GemmParams {
 template <bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-            const __grid_constant__ CUtensorMap map_b_tail, const GemmParams p) {
+            const __grid_constant__ CUtensorMap map_b_tail, const __grid_constant__ CUtensorMap map_c,
+            const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const PipeSmem ps = carve_smem(smem_raw);
+    uint8_t* c_stage = ps.stage_a + EPI_STAGE_OFFSET;      // one 32 x 32 fp32 staging tile per epilogue warp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t T_live = live_tokens(p.d_T, p.T_max);
     if (p.t0 >= T_live) return;
@@ -407,36 +409,34 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
-            const int row = (int)(item / n_tiles) * BM + quarter * 32 + lane;
             const int col0 = (int)(item % n_tiles) * BN;
             ok = mbar_wait(&ps.acc_full[acc], acc_phase, ps.abort_flag);
             ok = __all_sync(0xffffffffu, ok) != 0;
             if (!ok) break;
             tcgen05_fence_after();
-            float* crow = p.C + (int64_t)row * p.ldc;
+            // The warp's 32 rows x 32 columns leave through shared memory (128-byte swizzle) as one TMA tile store, or
+            // as one TMA reduction (global += tile) when the result is accumulated: whole 128-byte lines, no read of C by
+            // the SM, and rows / columns past M / N are clipped by the copy.
+            uint8_t* stg = c_stage + (size_t)(warp - 2) * EPI_STAGE_TILE;
+            const int row0 = (int)(item / n_tiles) * BM + quarter * 32;
 #pragma unroll 1
             for (int piece = col_half * EPI_PIECES; piece < (col_half + 1) * EPI_PIECES; ++piece) {
                 const int pc0 = col0 + piece * 32;
                 if (pc0 >= p.N) break;
                 float v[32];
                 tcgen05_ld_32x32(tmem_base + lane_addr + acc * BN + piece * 32, v);
-                if (row < p.M) {
-                    if (pc0 + 32 <= p.N && (p.ldc & 3) == 0) {
-                        float4* dst = reinterpret_cast<float4*>(crow + pc0);
+                if (lane == 0) bulk_wait_read_all();          // the previous tile copy has read the staging tile
+                __syncwarp();
 #pragma unroll
-                        for (int q4 = 0; q4 < 8; ++q4) {
-                            float4 o = make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
-                            if (p.accumulate) {
-                                const float4 c = dst[q4];
-                                o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
-                            }
-                            dst[q4] = o;
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (pc0 + j < p.N) crow[pc0 + j] = p.accumulate ? crow[pc0 + j] + v[j] : v[j];
-                    }
+                for (int q4 = 0; q4 < 8; ++q4)
+                    *reinterpret_cast<float4*>(stg + lane * 128 + ((q4 ^ (lane & 7)) << 4)) =
+                        make_float4(v[4 * q4], v[4 * q4 + 1], v[4 * q4 + 2], v[4 * q4 + 3]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && row0 < p.M) {
+                    if (p.accumulate) tma_reduce_add_2d(&map_c, pc0, row0, stg);
+                    else tma_store_2d(&map_c, pc0, row0, stg);
+                    bulk_commit_group();
                 }
             }
             tcgen05_fence_before();
@@ -444,6 +444,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ C
             if (lane == 0) mbar_arrive(&ps.acc_empty[acc]);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        if (lane == 0) bulk_wait_all();       // the tile copies have completed before the block's shared memory goes
     }
     pipe_teardown(ps, tmem_base, p.d_status);
 }
@@ -482,7 +483,8 @@ int arrol_internal_gemm_tn(arrol_ctx* ctx, const void* A, int64_t lda, const voi
                            float* C, int64_t ldc, int accumulate, cudaStream_t s) {
     if (M <= 0 || N <= 0 || K <= 0 || lda % 8 != 0 || ldb % 8 != 0) return ARROL_ERR_UNSUPPORTED;
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    CUtensorMap map_a, map_b;
+    CUtensorMap map_a, map_b, map_c;
+    if (make_map_f32_tile(ctx, &map_c, C, (uint64_t)M, (uint64_t)N, (uint64_t)ldc) != ARROL_OK) return ARROL_ERR_CUDA;
     bool a3 = M % 64 == 0, b3 = N % 64 == 0;
     if (a3 && make_map_mn3d(ctx, &map_a, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM / 64) != ARROL_OK) a3 = false;
     if (b3 && make_map_mn3d(ctx, &map_b, B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, BN / 64) != ARROL_OK) b3 = false;
@@ -493,7 +495,7 @@ int arrol_internal_gemm_tn(arrol_ctx* ctx, const void* A, int64_t lda, const voi
     g.a3d = a3; g.b3d = b3; g.d_T = nullptr; g.T_max = 1; g.t0 = 0; g.d_status = ctx->d_status;
     const int64_t items = (int64_t)((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     gemm_kernel<true, true><<<(unsigned)(items < ctx->sm_count ? items : ctx->sm_count), NUM_THREADS, SMEM_BYTES, s>>>(
-        map_a, map_b, map_b, g);
+        map_a, map_b, map_b, map_c, g);
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
@@ -525,7 +527,7 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     __nv_bfloat16* dZ = reinterpret_cast<__nv_bfloat16*>(static_cast<uint8_t*>(workspace) + L.dz);
     uint16_t* Htail = reinterpret_cast<uint16_t*>(static_cast<uint8_t*>(workspace) + L.tail);
 
-    ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DZ_SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(dz_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     ARROL_CUDA_OK(cudaFuncSetAttribute(gemm_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
 
@@ -537,6 +539,8 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
     if (make_map(ctx, &map_w_k, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map_ld(ctx, &map_dz_k, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, BM) != ARROL_OK) return ARROL_ERR_CUDA;
     if (make_map_ld(ctx, &map_dz_st, dZ, TC, (uint64_t)V, (uint64_t)L.ldz, 32) != ARROL_OK) return ARROL_ERR_CUDA;   // store tiles
+    CUtensorMap map_dw;
+    if (make_map_f32_tile(ctx, &map_dw, dW, (uint64_t)V, (uint64_t)d, (uint64_t)d) != ARROL_OK) return ARROL_ERR_CUDA;
     bool d3 = d % 64 == 0, v3 = V % 64 == 0;
     if (d3 && (make_map_mn3d(ctx, &map_w_mn, W_vocab, (uint64_t)V, (uint64_t)d, (uint64_t)d, BN / 64) != ARROL_OK ||
                make_map_mn3d(ctx, &map_h_tail, Htail, (uint64_t)BK, (uint64_t)d, (uint64_t)d, BN / 64) != ARROL_OK))
@@ -569,21 +573,24 @@ extern "C" int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const 
         zp.dZ = dZ; zp.d_status = ctx->d_status;
         int64_t grid = (int64_t)(TC / BM) * splits;
         if (grid > ctx->sm_count) grid = ctx->sm_count;
-        dz_kernel<<<(unsigned)grid, NUM_THREADS, DZ_SMEM_BYTES, s>>>(map_h_k, map_w_k, map_dz_st, zp);
+        dz_kernel<<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h_k, map_w_k, map_dz_st, zp);
 
         GemmParams gh;    // dH[chunk] = dZ . W
         gh.M = (int)rows; gh.N = d; gh.K = V; gh.C = dH + t0 * d; gh.ldc = d; gh.accumulate = 0; gh.k_is_tokens = 0; gh.a3d = 0; gh.b3d = d3;
         gh.d_T = d_T; gh.T_max = T_max; gh.t0 = t0; gh.d_status = ctx->d_status;
         const int64_t gh_items = (int64_t)((rows + BM - 1) / BM) * ((d + BN - 1) / BN);
+        CUtensorMap map_dh;      // this chunk's rows of dH: rows past the chunk are clipped by the tile stores
+        if (make_map_f32_tile(ctx, &map_dh, dH + t0 * d, (uint64_t)rows, (uint64_t)d, (uint64_t)d) != ARROL_OK)
+            return ARROL_ERR_CUDA;
         gemm_kernel<false, true><<<(unsigned)(gh_items < ctx->sm_count ? gh_items : ctx->sm_count), NUM_THREADS,
-                                   SMEM_BYTES, s>>>(map_dz_k, map_w_mn, map_w_mn, gh);
+                                   SMEM_BYTES, s>>>(map_dz_k, map_w_mn, map_w_mn, map_dh, gh);
         tail_block_kernel<<<64, 256, 0, s>>>(static_cast<const uint16_t*>(hidden), d, d_T, T_max, t0, Htail);
         GemmParams gw;    // dW += dZ^T . H[chunk]
         gw.M = V; gw.N = d; gw.K = (int)rows; gw.C = dW; gw.ldc = d; gw.accumulate = 1; gw.k_is_tokens = 1; gw.a3d = v3; gw.b3d = d3;
         gw.d_T = d_T; gw.T_max = T_max; gw.t0 = t0; gw.d_status = ctx->d_status;
         const int64_t gw_items = (int64_t)((V + BM - 1) / BM) * ((d + BN - 1) / BN);
         gemm_kernel<true, true><<<(unsigned)(gw_items < ctx->sm_count ? gw_items : ctx->sm_count), NUM_THREADS,
-                                  SMEM_BYTES, s>>>(map_dz_mn, map_h_mn, map_h_tail, gw);
+                                  SMEM_BYTES, s>>>(map_dz_mn, map_h_mn, map_h_tail, map_dw, gw);
         ctx->launches += 4;
         ARROL_CUDA_OK(cudaGetLastError());
     }
