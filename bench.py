@@ -408,6 +408,7 @@ def run_ours(args, w):
             "prune_step_us": prune_us,
             "compact_roofline": {"bound": "hbm", "achieved": compact_gbs, "peak": float(peaks["hbm_gbs"]),
                                  "unit": "GB/s", "frac": compact_gbs / float(peaks["hbm_gbs"]),
+                                 "frac_of_nominal_8000": compact_gbs / 8000.0,
                                  "algorithmic_bytes_per_launch": gather_bytes},
         }
         esz = pr.hidden_score.element_size()
@@ -415,7 +416,8 @@ def run_ours(args, w):
             gbs = n_score * w.d * esz / (score_ms * 1e-3) / 1e9
             out["score_roofline"] = {"kernel": "score_linear_kernel", "bound": "hbm", "rows": int(n_score),
                                      "achieved": gbs, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
-                                     "frac": gbs / float(peaks["hbm_gbs"]), "launch_ms": score_ms,
+                                     "frac": gbs / float(peaks["hbm_gbs"]), "frac_of_nominal_8000": gbs / 8000.0,
+                                     "launch_ms": score_ms,
                                      "note": "linear head streamed over consecutive source rows; the step itself "
                                              "scores only N = %d rows (launch-latency bound)" % w_rank.N}
         else:
