@@ -332,6 +332,39 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     score_ms = a.elapsed_time(b) / K
     del so
+    # the step's own scoring call (N rows) next to a copy of the same number of bytes: at this size both sit on the
+    # launch floor, which is the achievable roof there
+    step_score = None
+    if w.h == 0:
+        N_step = w_rank.N
+        so = [torch.empty(N_step, dtype=torch.float32, device=pr.dev) for _ in range(3)]
+        src = torch.empty((N_step, w.d), dtype=pr.hidden_score.dtype, device=pr.dev)
+        dst = torch.empty_like(src)
+        reps = max(K, 50)
+
+        def timed_us(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            for _ in range(8):            # device-side filler, so that the timed calls are queued behind it and the
+                filler()                  # host's launch time does not show
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps * 1e3
+
+        big = [torch.empty(n_score, dtype=torch.float32, device=pr.dev) for _ in range(3)]
+        filler = lambda: B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, n_score, big[0], big[1], big[2],
+                                               q_lut=pr.q_lut)
+        us_score = timed_us(lambda: B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, N_step, so[0], so[1], so[2],
+                                                          row_index=pr.row_index, q_lut=pr.q_lut))
+        us_copy = timed_us(lambda: dst.copy_(src))
+        step_score = {"rows": int(N_step), "bytes": int(N_step * w.d * src.element_size()), "us": us_score,
+                      "size_matched_copy_us": us_copy,
+                      "note": "device time of queued calls; the copy moves the same bytes once (read + write)"}
+        del so, src, dst, big
 
     # ---- policy update on the same survivors (reported separately; not part of `value`) ----
     update = None
@@ -419,7 +452,8 @@ def run_ours(args, w):
                                      "frac": gbs / float(peaks["hbm_gbs"]), "frac_of_nominal_8000": gbs / 8000.0,
                                      "launch_ms": score_ms,
                                      "note": "linear head streamed over consecutive source rows; the step itself "
-                                             "scores only N = %d rows (launch-latency bound)" % w_rank.N}
+                                             "scores only N = %d rows (launch-latency bound)" % w_rank.N,
+                                     "step_call": step_score}
         else:
             tfs = 2.0 * n_score * w.d * w.h / (score_ms * 1e-3) / 1e12
             tc_peak = float(peaks["bf16_tflops"])
