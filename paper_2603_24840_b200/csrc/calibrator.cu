@@ -206,33 +206,51 @@ calib_update_kernel(uint8_t* state, CalibLayout L, const int32_t* __restrict__ b
     }
     __syncthreads();
 
-    // delta: 64 bisection steps on E[p](delta) = kappa, by the first warp alone (no block barriers in the loop).  Per
-    // step the lanes form the per-bin products c_b p_b and lane 0 adds them in index order (the same rounding
-    // sequence as a plain loop: an empty bin adds exactly zero), so only the chain of B additions is serial.
+    // delta: 64 bisection steps on E[p](delta) = kappa, by the first warp alone (no block barriers in the loop).  The
+    // value that decides a step is the expected keep rate summed over the bins in index order, one rounding per
+    // operation (so that delta agrees bit for bit with a plain loop).  Per step the lanes form the per-bin products
+    // c_b p_b (all >= 0) and a butterfly sum S of them; the in-order sum differs from S by at most
+    // (B + 8) 2^-53 S (both are within their standard error bounds of the exact sum), so when S / n is further from
+    // kappa than four times that bound plus the rounding of the division, S / n < kappa already is the decision.
+    // Only the steps near convergence (about the last twenty) need the serial chain of B additions.
     if (wid == 0) {
         __shared__ double prod[MAX_BINS];
         const double n = __dadd_rn(n_pos, n_neg);
         double delta = 0.0;
         if (n > 0.0) {                                   // uniform for the warp
             double lo = -(1.0 + lambda), hi = 1.0 + lambda;
+            const double u = 1.1102230246251565e-16;     // 2^-53
             for (int it = 0; it < 64; ++it) {
                 const double mid = __dmul_rn(0.5, __dadd_rn(lo, hi));
                 const double base = __dadd_rn(kappa, mid);
+                double part = 0.0;
                 for (int b = lane; b < B; b += 32) {
                     double p = __dadd_rn(base, term[b]);
                     if (p < p_min) p = p_min;
                     if (p > p_max) p = p_max;
-                    prod[b] = __dmul_rn(weight[b], p);
+                    const double x = __dmul_rn(weight[b], p);
+                    prod[b] = x;
+                    part += x;
                 }
-                __syncwarp();
-                int below = 0;
-                if (lane == 0) {
-                    double e = 0.0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);   // the same bits in every lane
+                const double e_tree = part / n;
+                const double slack = 4.0 * ((double)(B + 8) * u * e_tree + 2.0 * u * (e_tree + kappa));
+                int below;
+                if (fabs(e_tree - kappa) > slack) {
+                    below = e_tree < kappa ? 1 : 0;
+                } else {
+                    __syncwarp();
+                    below = 0;
+                    if (lane == 0) {
+                        double e = 0.0;
 #pragma unroll 8
-                    for (int b = 0; b < B; ++b) e = __dadd_rn(e, prod[b]);
-                    below = __ddiv_rn(e, n) < kappa ? 1 : 0;
+                        for (int b = 0; b < B; ++b) e = __dadd_rn(e, prod[b]);
+                        below = __ddiv_rn(e, n) < kappa ? 1 : 0;
+                    }
+                    below = __shfl_sync(0xffffffffu, below, 0);
                 }
-                below = __shfl_sync(0xffffffffu, below, 0);       // also orders the reads of prod before the next writes
+                __syncwarp();                            // prod is rewritten by the next step
                 if (below) lo = mid; else hi = mid;
             }
             delta = __dmul_rn(0.5, __dadd_rn(lo, hi));

@@ -54,6 +54,34 @@ def test_calibrator_update_matches_oracle(ctx, n_bins, cap, sizes):
     assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
 
 
+def test_delta_is_bit_equal_over_many_states_and_parameters(ctx):
+    """delta decides by comparisons that turn on the last bits near convergence: many random buffer states, skewed
+    score distributions and survival parameters, every one bit for bit."""
+    g = np.random.default_rng(77)
+    params = [(0.5, 0.5, 0.5, 0.05, 0.95), (0.25, 1.0, 0.3, 0.0, 1.0), (0.75, 0.2, 0.6, 0.1, 0.9), (0.5, 0.0, 0.5, 0.0, 1.0),
+              (0.9, 2.0, 0.5, 0.05, 0.95), (0.1, 0.5, 0.9, 0.0, 0.5)]
+    for case in range(36):
+        kappa, lam, rho, pmin, pmax = params[case % len(params)]
+        n_bins = [128, 128, 16, 64, 5, 128][case % 6]
+        cap = [8192, 300, 64, 1000, 50, 2048][(case // 2) % 6]
+        cal = CAL.Calibrator(ctx, n_bins, cap, alpha=1.0)
+        buf = oracle.ScoreBuffers(cap)
+        sp = CAL.survival(kappa, lam, rho, pmin, pmax)
+        a, b = [(2, 2), (0.5, 0.5), (8, 1), (1, 8), (5, 5), (0.3, 3)][case % 6]
+        for n in (int(g.integers(1, 3000)), int(g.integers(1, 500))):
+            prob = g.beta(a, b, size=n).astype(np.float32)
+            rew = (g.random(n) < prob ** [1.0, 0.3, 3.0][case % 3]).astype(np.float32)
+            bins = np.array([oracle.bin_index(float(v), n_bins) for v in prob], dtype=np.int32)
+            cal.update(torch.from_numpy(bins).cuda(), torch.from_numpy(rew).cuda(), sp)
+            buf.push(prob.astype(np.float64), rew > 0.5)
+            torch.cuda.synchronize()
+            cpos, cneg = buf.counts(n_bins)
+            _, lut = oracle.build_q_lut(cpos, cneg, 1.0)
+            delta = oracle.solve_delta(cpos, cneg, lut, kappa, lam, rho, pmin, pmax, iters=64)
+            assert cal.snapshot()["delta"] == delta, (case, n)
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
+
+
 def test_stochastic_selection_matches_oracle(ctx):
     g = np.random.default_rng(5)
     N = 100003
