@@ -71,3 +71,27 @@ def test_create_without_a_device_fails_loudly(lib):
     assert rc in (-7, -5) and not h.value          # no CPU fallback: the context cannot be made
     with pytest.raises(B.ArrolError):
         B.Context(0)
+
+
+def test_header_is_plain_c_and_links_against_the_library(tmp_path, lib):
+    """The boundary is a C ABI: the header compiles as strict C99 and a C program links against the library and
+    calls an entry point that needs no GPU."""
+    import os
+    import shutil
+    import subprocess
+    from paper_2603_24840_b200 import binding as B
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "c_abi.c"
+    src.write_text('#include <stdio.h>\n#include "arrol.h"\n'
+                   'int main(void) { printf("%d %s\\n", arrol_version(), arrol_status_string(ARROL_ERR_WORKSPACE));\n'
+                   '  return arrol_create(NULL, 0) == ARROL_ERR_INVALID_ARG ? 0 : 1; }\n')
+    exe = tmp_path / "c_abi"
+    libdir = os.path.dirname(B.LIB_PATH)
+    subprocess.check_call([gcc, "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(root, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-l:libarrol.so", "-Wl,-rpath," + libdir])
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0
+    assert out.stdout.split()[0] == str(B.arrol_version())
