@@ -324,13 +324,17 @@ def run_ours(args, w):
         B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, n_score, so[0], so[1], so[2], row_index=ridx,
                               q_lut=pr.q_lut)
     torch.cuda.synchronize()
+    reps_score = K if w.h == 0 else max(K, 20)
+    if w.h:                    # a call of tens of microseconds: queue it behind device work so that the host's
+        for _ in range(2):     # launch time does not show
+            pr.compact()
     a.record(stream)
-    for _ in range(K):
+    for _ in range(reps_score):
         B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, n_score, so[0], so[1], so[2], row_index=ridx,
                               q_lut=pr.q_lut)
     b.record(stream)
     torch.cuda.synchronize()
-    score_ms = a.elapsed_time(b) / K
+    score_ms = a.elapsed_time(b) / reps_score
     del so
     # the step's own scoring call (N rows) next to a copy of the same number of bytes: at this size both sit on the
     # launch floor, which is the achievable roof there
