@@ -2,7 +2,10 @@
  * CPU oracle: trace confidence (Section 3 "Trace Confidence").  TEST INFRASTRUCTURE ONLY (see arrol_oracle.c).
  *   token confidence   H_t = - sum_{j=1..V} log P_t(j),  P_t = softmax of the position's logits
  *   window confidence  H_w = mean of H_t over a sliding window of `window` tokens
- *   trace score        mode 0: mean of H_t over the trace;  mode 1: minimum window confidence over the trace
+ *   trace score        mode 0: mean of H_t over the trace;  mode 1: minimum window confidence over the trace;
+ *                      mode 2: average of the bottom 10 % of the window confidences: the windows are all
+ *                      len - w + 1 sliding positions, the k = ceil(0.1 * #windows) smallest H_w are averaged
+ *                      (at least one window, so a trace with fewer than ten windows gives its minimum)
  * A trace shorter than the window has one window, the whole trace.
  */
 #include <math.h>
@@ -52,6 +55,11 @@ int oracle_token_confidence(const void* hidden, const void* W, int dtype, const 
     return err;
 }
 
+static int cmp_double(const void* a, const void* b) {
+    const double x = *(const double*)a, y = *(const double*)b;
+    return (x > y) - (x < y);
+}
+
 void oracle_trace_confidence(const double* H, const int64_t* cu_seqlens, int64_t S, int window, int mode, double* out) {
     for (int64_t s = 0; s < S; ++s) {
         const int64_t t0 = cu_seqlens[s], len = cu_seqlens[s + 1] - t0;
@@ -60,6 +68,22 @@ void oracle_trace_confidence(const double* H, const int64_t* cu_seqlens, int64_t
             double sum = 0.0;
             for (int64_t t = 0; t < len; ++t) sum = sum + H[t0 + t];
             out[s] = sum / (double)len;
+        } else if (mode == 2) {
+            const int64_t w = len < window ? len : window;
+            const int64_t n_win = len - w + 1;
+            double* hw = (double*)malloc(sizeof(double) * (size_t)n_win);
+            if (!hw) { out[s] = NAN; continue; }
+            for (int64_t a = 0; a < n_win; ++a) {
+                double sum = 0.0;
+                for (int64_t t = 0; t < w; ++t) sum = sum + H[t0 + a + t];
+                hw[a] = sum / (double)w;
+            }
+            qsort(hw, (size_t)n_win, sizeof(double), cmp_double);
+            const int64_t k = (n_win + 9) / 10;
+            double sum = 0.0;
+            for (int64_t a = 0; a < k; ++a) sum = sum + hw[a];
+            out[s] = sum / (double)k;
+            free(hw);
         } else {
             const int64_t w = len < window ? len : window;
             double best = INFINITY;

@@ -49,3 +49,33 @@ def test_trace_confidence_brute_force():
             assert abs(mn[s] - expect) < 1e-10
     # window 1 is the minimum token confidence; a window as long as the trace is the mean
     assert np.allclose(oc.trace_confidence(Hs, cu, window=1, mode=1)[[0, 1, 3]], [Hs[0], Hs[1:6].min(), Hs[6:23].min()])
+
+
+def test_bottom_tenth_of_the_windows_brute_force():
+    """mode 2: mean of the ceil(0.1 n) lowest window means, against a Python sort; hand-worked cases."""
+    g = np.random.default_rng(2)
+    ell = np.array([1, 9, 10, 11, 0, 25, 137, 64])
+    cu = np.concatenate([[0], np.cumsum(ell)])
+    Hs = g.random(int(cu[-1])) * 100
+    for w in (1, 3, 16, 1000):
+        got = oc.trace_confidence(Hs, cu, window=w, mode=2)
+        mn = oc.trace_confidence(Hs, cu, window=w, mode=1)
+        for s, n in enumerate(ell):
+            seg = Hs[cu[s]:cu[s + 1]]
+            if n == 0:
+                assert got[s] == 0.0
+                continue
+            ww = min(w, n)
+            means = sorted(seg[a:a + ww].mean() for a in range(n - ww + 1))
+            k = -(-len(means) // 10)
+            assert abs(got[s] - sum(means[:k]) / k) < 1e-10
+            assert got[s] >= mn[s] - 1e-12
+            if len(means) <= 10:                      # one window in the bottom tenth: the minimum itself
+                assert abs(got[s] - mn[s]) < 1e-12
+    # by hand: H = 1..20, window 1: 20 windows, bottom 10 % = the two smallest = (1 + 2) / 2
+    H = np.arange(1.0, 21.0)[::-1].copy()
+    assert oc.trace_confidence(H, np.array([0, 20]), window=1, mode=2)[0] == 1.5
+    # window 2 on 1..21 ascending: 20 window means 1.5, 2.5, ...: bottom two average to 2.0
+    assert oc.trace_confidence(np.arange(1.0, 22.0), np.array([0, 21]), window=2, mode=2)[0] == 2.0
+    # 11 windows -> k = 2 (ceil), not 1 (floor)
+    assert oc.trace_confidence(np.arange(1.0, 12.0), np.array([0, 11]), window=1, mode=2)[0] == 1.5
