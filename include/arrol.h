@@ -50,20 +50,24 @@ typedef enum {
 #define ARROL_DEV_CAPACITY 1u      /* arrol_compact: T > dst_capacity_tokens, nothing was gathered */
 #define ARROL_DEV_BAD_TARGET 2u    /* arrol_token_logprob: a target id >= V (its logp is set to 0) */
 #define ARROL_DEV_WAIT_EXPIRED 4u  /* arrol_token_logprob: a pipeline wait hit its iteration limit */
+#define ARROL_DEV_BAD_STATE 8u     /* arrol_calib_update: the state's header does not match (B, cap); state untouched */
+#define ARROL_DEV_BAD_INDEX 16u    /* a source row outside the bound set with arrol_set_source_rows; access skipped */
 
 int arrol_version(void);                    /* major*10000 + minor*100 + patch */
 const char* arrol_status_string(int status); /* static string, never NULL */
 
 /* Creates a context on CUDA device `device` (made current for the calling thread during the call).
  * Allocates the context's device status word, a 16 MB scratch buffer and a 64 MB row-packing buffer (MLP head),
- * 1 MB of pinned host memory, a second stream and a few events (used by arrol_prune_rebatch_host); nothing is
+ * 65 MB of pinned host memory, a second stream and a few events (used by arrol_prune_rebatch_host); nothing is
  * allocated later.  Calls that use the context's buffers (MLP-head scoring, the policy loss, the head training
  * step) must be ordered on the device with respect to one another, e.g. by issuing them on one stream. */
 int arrol_create(arrol_ctx** out, int device);
 int arrol_destroy(arrol_ctx* ctx);
 
 /* Waits for `stream`, copies the device status word to *dev_status_bits (host pointer, may be NULL),
- * clears it, and returns ARROL_OK if it was 0, else ARROL_ERR_CAPACITY / ARROL_ERR_DEVICE_STATUS. */
+ * clears it, and returns ARROL_OK if it was 0, else ARROL_ERR_CAPACITY / ARROL_ERR_DEVICE_STATUS.
+ * Order it after all work on the context: the word is read and then cleared on `stream`, so a bit that a kernel on
+ * another stream sets between the two is lost. */
 int arrol_poll_status(arrol_ctx* ctx, void* stream, uint32_t* dev_status_bits);
 
 /* ---- Binned posterior table: host helpers (Appendix A.4).  All pointers are HOST pointers. ----------
@@ -209,6 +213,8 @@ int arrol_prune_step(arrol_ctx* ctx, const arrol_prune_step_args* args, void* st
  *   and solves delta by 64 bisection steps on [-(1+lambda), 1+lambda] so that
  *     sum_b (c_b^+ + c_b^-) clip(kappa + delta + lambda (rho - q_b), p_min, p_max) / (n+ + n-) = kappa
  *   (delta = 0 while both rings are empty).  fp64, one rounding per operation, fixed order: reproducible bit for bit.
+ *   (B, cap) must be the pair the state was initialised with: otherwise the state is left untouched and
+ *   ARROL_DEV_BAD_STATE is recorded.
  * arrol_calib_q_lut / arrol_calib_delta: device addresses of the table and of delta inside the state (pointer
  *   arithmetic on the host; no device access), to be passed to arrol_score_partial / arrol_select_stochastic.
  * arrol_calib_layout: byte offsets {c+, c-, q_lut, ring+, ring-, total} inside the state, for inspection.
@@ -270,8 +276,11 @@ int arrol_lm_head_backward(arrol_ctx* ctx, const void* hidden, const void* W_voc
  * arrol_trace_confidence: per packed trace s < S (S read from d_num = {S, T}; bounds from cu_seqlens):
  *     mode 0: trace_conf[s] = mean of token_conf over the trace;
  *     mode 1: trace_conf[s] = minimum over the trace of the mean of token_conf over a sliding window of `window`
- *             tokens (a trace shorter than the window has one window, the whole trace).
- *   An empty trace gives 0.  trace_conf float [S_max].  fp64 accumulation. */
+ *             tokens (a trace shorter than the window has one window, the whole trace);
+ *     mode 2: trace_conf[s] = mean of the lowest ceil(0.1 n) of the n = len - window + 1 sliding-window means (the
+ *             "bottom 10 % of the windows"; fewer than ten windows give the minimum).
+ *   An empty trace gives 0.  trace_conf float [S_max]; cu_seqlens holds at least S_max + 1 entries; S is clamped to
+ *   S_max, so a count in d_num larger than the arrays is never followed.  fp64 accumulation. */
 int arrol_token_logprob_conf(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
                              int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                              float* logp, float* lse, float* token_conf, void* workspace, size_t workspace_bytes,
@@ -309,17 +318,19 @@ int arrol_rank_vote(arrol_ctx* ctx, const float* score, const int32_t* answer, i
 
 /* ---- Whole step from host buffers (Algorithm 1, frontend lines "filter ... rebatch ... log-probs on R'") --
  * Convenience call for callers whose per-step data lives in host memory.  Only what the step needs is uploaded:
- * the small per-rollout arrays and token ids, the N hidden rows at the detection length (each to its own place in
- * d_hidden, for the head), and - once arrol_score_partial and arrol_select have produced the keep mask, which is
- * read back to plan the copies - the survivors' hidden rows, copied straight into their packed positions in
- * d_dst_rows.  arrol_compact then produces the scan, advantages and packed token ids, and arrol_token_logprob runs
+ * the small per-rollout arrays, the N hidden rows at the detection length (gathered into a pinned staging block of
+ * the context and sent as one copy into d_hidden as a packed [N, d] block, for the head), and - once
+ * arrol_score_partial and arrol_select have produced the keep mask, which is read back to plan the copies - the
+ * survivors' hidden rows and token ids, copied straight into their packed positions in d_dst_rows / d_dst_tokens.
+ * arrol_compact then produces the scan and the advantages, and arrol_token_logprob runs
  * per chunk of tokens as soon as the chunk's rows have landed (uploads on the context's second stream overlap the
  * tensor-core work).  Results are copied back and the stream is synchronised: the call is synchronous (one
  * synchronisation in the middle, one at the end) and allocates no device memory.
  * The quality head reads, for rollout i, source row src_tok_off[i] + cutoff - 1 (its hidden state at the
  * detection length).  Pointers prefixed h_ are HOST pointers (pinned memory gives full copy speed and real overlap),
  * d_ are DEVICE buffers provided by the caller with at least the stated sizes.  Model state (head, calib, W_vocab)
- * is device-resident.  P*G <= 1,048,576.  After the call only the scored rows of d_hidden are defined. */
+ * is device-resident.  P*G <= 1,048,576; head.d must equal d, d % 8 == 0; the workspace must be 256-byte aligned and
+ * large enough (ARROL_ERR_WORKSPACE before anything is copied).  After the call d_hidden holds the N scored rows. */
 typedef struct arrol_host_step {
     int32_t P, G, K, cutoff;       /* prompts, group size, survivors per group, detection length (>= 1)         */
     int32_t d, V;                  /* hidden width, vocabulary                                                  */
@@ -339,11 +350,11 @@ typedef struct arrol_host_step {
     arrol_calib calib;
     const void* W_vocab;           /* [V, d] bf16                                                               */
     /* staging and outputs, device */
-    void* d_hidden;                /* [T_src, d] bf16                                                           */
-    int32_t* d_src_tokens;         /* [T_src]                                                                   */
+    void* d_hidden;                /* [P*G, d] bf16: receives the scored rows                                   */
+    int32_t* d_src_tokens;         /* unused (may be NULL): token ids are uploaded packed into d_dst_tokens     */
     int32_t* d_lengths;            /* [P*G]                                                                     */
     int64_t* d_src_tok_off;        /* [P*G]                                                                     */
-    int64_t* d_row_index;          /* [P*G]                                                                     */
+    int64_t* d_row_index;          /* unused (may be NULL)                                                      */
     float* d_rewards;              /* [P*G]                                                                     */
     float *d_score, *d_prob, *d_q; /* [P*G] each                                                                */
     uint8_t* d_keep;               /* [P*G]                                                                     */
@@ -394,6 +405,18 @@ int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* step, void* 
 int arrol_score_partial_static(const void* hidden, int64_t row_stride_elems, const int64_t* row_index, int32_t N,
                                const arrol_head* head, const arrol_calib* calib, float* score, float* prob,
                                int32_t* bin, float* q, void* stream);
+
+/* ---- Index checks on request (no counterpart in the paper) -----------------------------------------------------
+ * The compute calls trust row_index and src_tok_off + lengths, because their signatures carry no size of the source
+ * buffers.  After arrol_set_source_rows(ctx, R) with R > 0 (the number of rows of `hidden` / src_tokens / src_rows),
+ * every call on the context checks them on the device instead of following them:
+ *   arrol_score_partial / arrol_prune_step: a row number outside [0, R) is never read; that rollout is scored as if
+ *     its hidden row were zero;
+ *   arrol_compact: if any kept rollout has src_tok_off < 0 or src_tok_off + length > R, the scan outputs are written
+ *     and nothing is gathered (as for a capacity overflow);
+ * and ARROL_DEV_BAD_INDEX is recorded in the status word.  R = 0 (the default) switches the checks off.  The other
+ * calls (arrol_head_grad, arrol_token_logprob, ...) are not covered. */
+int arrol_set_source_rows(arrol_ctx* ctx, int64_t source_rows);
 
 /* Number of kernels this context has launched so far (host-side count; -1 for a NULL context). */
 int64_t arrol_launch_count(arrol_ctx* ctx);

@@ -26,7 +26,7 @@ EXPORTS = [
     "arrol_calib_delta", "arrol_select_stochastic",
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
     "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
-    "arrol_prune_step", "arrol_token_logprob_splits", "arrol_test_hook",
+    "arrol_prune_step", "arrol_token_logprob_splits", "arrol_test_hook", "arrol_set_source_rows",
 ]
 
 
@@ -281,6 +281,13 @@ def arrol_test_hook(ctx: Context, key: int, value: int):
     lib = load_library()
     lib.arrol_test_hook.argtypes = [C.c_void_p, C.c_int32, C.c_int64]
     _check(lib.arrol_test_hook(ctx.handle, int(key), int(value)), "arrol_test_hook")
+
+
+def arrol_set_source_rows(ctx: Context, source_rows: int):
+    """Switches on (source_rows > 0) or off (0) the device-side range checks of row_index / src_tok_off + lengths."""
+    lib = load_library()
+    lib.arrol_set_source_rows.argtypes = [C.c_void_p, C.c_int64]
+    _check(lib.arrol_set_source_rows(ctx.handle, int(source_rows)), "arrol_set_source_rows")
 
 
 def arrol_launch_count(ctx: Context) -> int:

@@ -7,6 +7,7 @@
 
 constexpr int ARROL_COPY_EVENTS = 64;
 constexpr int ARROL_MAX_HOST_N = 1 << 20;   // rollouts per arrol_prune_rebatch_host call
+constexpr size_t ARROL_STAGE_BYTES = (size_t)64 << 20;
 
 struct arrol_ctx {
     int device;
@@ -25,6 +26,8 @@ struct arrol_ctx {
     cudaStream_t copy_stream;      // second stream of the host-buffer step: uploads overlap the log-prob kernel
     cudaEvent_t copy_events[ARROL_COPY_EVENTS];
     uint8_t* h_keep;               // pinned, ARROL_MAX_HOST_N bytes: the keep mask read back by the host-buffer step
+    int64_t source_rows;           // arrol_set_source_rows: rows of the caller's source buffers, 0 = indices unchecked
+    uint8_t* h_stage;              // pinned, ARROL_STAGE_BYTES: the scored rows of the host-buffer step, packed for one copy
 };
 
 constexpr int ARROL_MAX_MLP_N = 65536;       // rollouts per arrol_score_partial call with an MLP head

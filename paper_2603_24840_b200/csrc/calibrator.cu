@@ -71,8 +71,14 @@ __global__ void calib_init_kernel(uint8_t* state, int B, int64_t cap, double alp
 __global__ void __launch_bounds__(CAL_THREADS)
 calib_update_kernel(uint8_t* state, CalibLayout L, const int32_t* __restrict__ bin, const float* __restrict__ rewards,
                     const uint8_t* __restrict__ mask, int N, double kappa, double lambda, double rho, double p_min,
-                    double p_max) {
+                    double p_max, int B_arg, int64_t cap_arg, uint32_t* d_status) {
     CalibHeader* hd = reinterpret_cast<CalibHeader*>(state);
+    // The byte layout L comes from the call's (B, cap); the state must have been initialised with the same pair.
+    // A mismatched or uninitialised state is left untouched and reported (uniform over the block: no barrier yet).
+    if (hd->B != B_arg || hd->cap != cap_arg) {
+        if (threadIdx.x == 0) atomicOr(d_status, ARROL_DEV_BAD_STATE);
+        return;
+    }
     int64_t* cnt[2] = {reinterpret_cast<int64_t*>(state + L.cneg), reinterpret_cast<int64_t*>(state + L.cpos)};
     int16_t* ring[2] = {reinterpret_cast<int16_t*>(state + L.ring_neg), reinterpret_cast<int16_t*>(state + L.ring_pos)};
     float* lut = reinterpret_cast<float*>(state + L.q_lut);
@@ -334,7 +340,7 @@ extern "C" int arrol_calib_update(arrol_ctx* ctx, void* state, int32_t B, int64_
     if (!guard.ok) return ARROL_ERR_CUDA;
     calib_update_kernel<<<1, CAL_THREADS, 0, (cudaStream_t)stream>>>(static_cast<uint8_t*>(state), layout_of(B, cap), bin,
                                                                   rewards, mask, N, sp->kappa, sp->lambda, sp->rho,
-                                                                  sp->p_min, sp->p_max);
+                                                                  sp->p_min, sp->p_max, B, cap, ctx->d_status);
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;

@@ -23,7 +23,8 @@ __global__ void __launch_bounds__(SCAN_THREADS)
 scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ lengths, int N, int G,
                 const float* __restrict__ rewards, double eps, int ddof, int64_t capacity,
                 int32_t* __restrict__ survivor_idx, int64_t* __restrict__ cu_seqlens, float* __restrict__ adv,
-                int64_t* __restrict__ d_num, uint32_t* __restrict__ d_status) {
+                int64_t* __restrict__ d_num, uint32_t* __restrict__ d_status,
+                const int64_t* __restrict__ src_tok_off, int64_t source_rows) {
     __shared__ int32_t warp_cnt[32];
     __shared__ int64_t warp_tok[32];
     // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them)
@@ -37,7 +38,9 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
     pdl_launch_dependents();
     pdl_wait();
     keep = pdl_acquire(keep); lengths = pdl_acquire(lengths); rewards = pdl_acquire(rewards);
+    src_tok_off = pdl_acquire(src_tok_off);
     if (threadIdx.x == 0) cu_seqlens[0] = 0;
+    bool bad_index = false;          // a kept rollout whose source rows leave the caller's buffer (checked on request)
     int32_t carry_c = 0;             // survivors / tokens of the passes so far (the same in every thread)
     int64_t carry_t = 0;
 
@@ -125,6 +128,10 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
         for (int u = 0; u < SCAN_ITEMS; ++u) {
             kept[u] = s_keep[threadIdx.x * SCAN_ITEMS + u] != 0;
             if (!kept[u]) len[u] = 0;
+            else if (source_rows > 0) {
+                const int64_t o = src_tok_off[i0 + u];
+                bad_index = bad_index || o < 0 || o + len[u] > source_rows;
+            }
         }
         const int g_lo = base / G;
         if (shared_stats) {          // one thread per group of this pass; visible after the scan's first barrier
@@ -178,10 +185,13 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
         carry_t += pass_tok;
         __syncthreads();                 // the staging arrays and warp totals are rewritten by the next pass
     }
+    const int any_bad = __syncthreads_or(bad_index ? 1 : 0);
     if (threadIdx.x == 0) {
         d_num[0] = carry_c;
         d_num[1] = carry_t;
         if (carry_t > capacity) atomicOr(d_status, ARROL_DEV_CAPACITY);
+        if (any_bad) atomicOr(d_status, ARROL_DEV_BAD_INDEX);
+        d_status[1] = any_bad ? 1u : 0u;       // gate word: the gather kernels of this call copy nothing when it is set
     }
 }
 
@@ -219,17 +229,18 @@ gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_
               const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
               const int32_t* __restrict__ src_tokens, const uint4* __restrict__ src_rows, int vec_per_row,
               const float* __restrict__ adv, int64_t capacity, int tile_rows, int32_t* __restrict__ dst_tokens,
-              uint4* __restrict__ dst_rows, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
+              uint4* __restrict__ dst_rows, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq,
+              const uint32_t* __restrict__ gate) {
     __shared__ int64_t src_row_of[MAX_TILE_ROWS];
     __shared__ int s_first[2];               // survivor of the first row of the current / next tile
     pdl_launch_dependents();
     pdl_wait();
     d_num = pdl_acquire(d_num); cu_seqlens = pdl_acquire(cu_seqlens); survivor_idx = pdl_acquire(survivor_idx);
     src_tok_off = pdl_acquire(src_tok_off); src_tokens = pdl_acquire(src_tokens); src_rows = pdl_acquire(src_rows);
-    adv = pdl_acquire(adv);
+    adv = pdl_acquire(adv); gate = pdl_acquire(gate);
     const int S = (int)d_num[0];
     const int64_t T = d_num[1];
-    if (T > capacity || S <= 0 || T <= 0) return;      // capacity overflow was recorded by the scan kernel
+    if (T > capacity || S <= 0 || T <= 0 || *gate) return;   // overflow / bad index was recorded by the scan kernel
     const int64_t n_tiles = (T + tile_rows - 1) / tile_rows;
     const int64_t tiles_per_block = (n_tiles + gridDim.x - 1) / gridDim.x;
     const int64_t tile_begin = (int64_t)blockIdx.x * tiles_per_block;
@@ -289,13 +300,15 @@ __global__ void __launch_bounds__(TOKENS_THREADS)
 gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_seqlens,
                      const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
                      const int32_t* __restrict__ src_tokens, const float* __restrict__ adv, int64_t capacity,
-                     int32_t* __restrict__ dst_tokens, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq) {
+                     int32_t* __restrict__ dst_tokens, float* __restrict__ tok_adv, int32_t* __restrict__ tok_seq,
+                     const uint32_t* __restrict__ gate) {
     pdl_launch_dependents();
     pdl_wait();
     d_num = pdl_acquire(d_num); cu_seqlens = pdl_acquire(cu_seqlens); survivor_idx = pdl_acquire(survivor_idx);
     src_tok_off = pdl_acquire(src_tok_off); src_tokens = pdl_acquire(src_tokens); adv = pdl_acquire(adv);
+    gate = pdl_acquire(gate);
     const int S = (int)d_num[0];
-    if (d_num[1] > capacity) return;                       // capacity overflow was recorded by the scan kernel
+    if (d_num[1] > capacity || *gate) return;              // overflow / bad index was recorded by the scan kernel
     for (int s = blockIdx.x; s < S; s += gridDim.x) {
         const int64_t c0 = __ldg(cu_seqlens + s);
         const int len = (int)(__ldg(cu_seqlens + s + 1) - c0);
@@ -346,7 +359,7 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     cudaStream_t s = (cudaStream_t)stream;
     ARROL_CUDA_OK(arrol_launch_pdl(scan_adv_kernel, dim3(1), dim3(SCAN_THREADS), 0, s, keep, lengths, N, G, rewards,
                                    (double)eps, ddof, dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
-                                   ctx->d_status));
+                                   ctx->d_status, src_tok_off, ctx->source_rows));
     ctx->launches += 1;
     const bool any_token_output = dst_tokens || dst_rows || tok_adv || tok_seq;
     if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
@@ -365,7 +378,7 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
         int64_t blocks = N < (int64_t)ctx->sm_count * 16 ? N : (int64_t)ctx->sm_count * 16;
         ARROL_CUDA_OK(arrol_launch_pdl(gather_tokens_kernel, dim3((unsigned)blocks), dim3(TOKENS_THREADS), 0, s, d_num,
                                        cu_seqlens, survivor_idx, src_tok_off, src_tokens, adv, dst_capacity_tokens,
-                                       dst_tokens, tok_adv, tok_seq));
+                                       dst_tokens, tok_adv, tok_seq, ctx->d_status + 1));
         ctx->launches += 1;
         return ARROL_OK;
     }
@@ -386,7 +399,7 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
     ARROL_CUDA_OK(arrol_launch_pdl(gather_kernel, dim3((unsigned)blocks), dim3(GATHER_THREADS), 0, s, d_num, cu_seqlens,
                                    survivor_idx, src_tok_off, src_tokens, static_cast<const uint4*>(src_rows),
                                    vec_per_row, adv, dst_capacity_tokens, tile_rows, dst_tokens,
-                                   static_cast<uint4*>(dst_rows), tok_adv, tok_seq));
+                                   static_cast<uint4*>(dst_rows), tok_adv, tok_seq, ctx->d_status + 1));
     ctx->launches += 1;
     return ARROL_OK;
 }

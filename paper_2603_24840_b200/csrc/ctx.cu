@@ -14,7 +14,7 @@ extern "C" const char* arrol_status_string(int status) {
         case ARROL_ERR_WORKSPACE: return "workspace missing or too small";
         case ARROL_ERR_CAPACITY: return "destination capacity exceeded (detected on the device)";
         case ARROL_ERR_CUDA: return "a CUDA call failed";
-        case ARROL_ERR_DEVICE_STATUS: return "device-detected error (bad target id or expired wait)";
+        case ARROL_ERR_DEVICE_STATUS: return "device-detected error (bad target id, expired wait, bad state or index)";
         case ARROL_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
         default: return "unknown status";
     }
@@ -52,6 +52,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->launches = 0;
     ctx->copy_stream = nullptr;
     ctx->h_keep = nullptr;
+    ctx->h_stage = nullptr;
+    ctx->source_rows = 0;
     for (int i = 0; i < ARROL_COPY_EVENTS; ++i) ctx->copy_events[i] = nullptr;
     bool ok = cudaMalloc(&ctx->d_status, 256) == cudaSuccess &&
               cudaMemset(ctx->d_status, 0, 256) == cudaSuccess &&
@@ -61,6 +63,7 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
               cudaMalloc(&ctx->d_tile_counters, ARROL_TILE_COUNTERS * sizeof(uint32_t)) == cudaSuccess &&
               cudaMemset(ctx->d_tile_counters, 0, ARROL_TILE_COUNTERS * sizeof(uint32_t)) == cudaSuccess &&
               cudaMallocHost(&ctx->h_keep, ARROL_MAX_HOST_N) == cudaSuccess &&
+              cudaMallocHost(&ctx->h_stage, ARROL_STAGE_BYTES) == cudaSuccess &&
               cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; ok && i < ARROL_COPY_EVENTS; ++i)
         ok = cudaEventCreateWithFlags(&ctx->copy_events[i], cudaEventDisableTiming) == cudaSuccess;
@@ -89,10 +92,17 @@ extern "C" int arrol_destroy(arrol_ctx* ctx) {
     if (ctx->d_pack) (void)cudaFree(ctx->d_pack);
     if (ctx->d_tile_counters) (void)cudaFree(ctx->d_tile_counters);
     if (ctx->h_keep) (void)cudaFreeHost(ctx->h_keep);
+    if (ctx->h_stage) (void)cudaFreeHost(ctx->h_stage);
     for (int i = 0; i < ARROL_COPY_EVENTS; ++i)
         if (ctx->copy_events[i]) (void)cudaEventDestroy(ctx->copy_events[i]);
     if (ctx->copy_stream) (void)cudaStreamDestroy(ctx->copy_stream);
     delete ctx;
+    return ARROL_OK;
+}
+
+extern "C" int arrol_set_source_rows(arrol_ctx* ctx, int64_t source_rows) {
+    if (!ctx || source_rows < 0) return ARROL_ERR_INVALID_ARG;
+    ctx->source_rows = source_rows;
     return ARROL_OK;
 }
 
@@ -124,7 +134,8 @@ extern "C" int arrol_poll_status(arrol_ctx* ctx, void* stream, uint32_t* dev_sta
     uint32_t bits = *ctx->h_status;
     if (dev_status_bits) *dev_status_bits = bits;
     if (bits == 0) return ARROL_OK;
-    if (bits & (ARROL_DEV_BAD_TARGET | ARROL_DEV_WAIT_EXPIRED)) return ARROL_ERR_DEVICE_STATUS;
+    if (bits & (ARROL_DEV_BAD_TARGET | ARROL_DEV_WAIT_EXPIRED | ARROL_DEV_BAD_STATE | ARROL_DEV_BAD_INDEX))
+        return ARROL_ERR_DEVICE_STATUS;
     return ARROL_ERR_CAPACITY;
 }
 

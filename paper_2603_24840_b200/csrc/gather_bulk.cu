@@ -63,7 +63,7 @@ gather_rows_bulk_kernel(const int64_t* __restrict__ d_num, const int64_t* __rest
 
     const int S = (int)d_num[0];
     const int64_t T = d_num[1];
-    if (T > capacity || S <= 0 || T <= 0) return;          // capacity overflow was recorded by the scan kernel
+    if (T > capacity || S <= 0 || T <= 0 || d_status[1]) return;   // overflow / bad index was recorded by the scan kernel
     const int64_t n_tiles = (T + tile_rows - 1) / tile_rows;
     const int64_t per_block = (n_tiles + gridDim.x - 1) / gridDim.x;
     const int64_t tile_begin = (int64_t)blockIdx.x * per_block;

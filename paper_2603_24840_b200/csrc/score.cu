@@ -60,7 +60,8 @@ template <typename T>
 __global__ void __launch_bounds__(128)
 score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index, int N,
                     int d, const T* __restrict__ w, const T* __restrict__ bias, int B,
-                    const float* __restrict__ q_lut, float* score, float* prob, int32_t* bin, float* q) {
+                    const float* __restrict__ q_lut, float* score, float* prob, int32_t* bin, float* q,
+                    int64_t source_rows, uint32_t* d_status) {
     constexpr int VN = Vec16<T>::N;
     pdl_launch_dependents();
     pdl_wait();
@@ -71,7 +72,11 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
     if (warp >= N) return;
     const int64_t row = row_index ? row_index[warp] : (int64_t)warp;
     const T* x = hidden + row * row_stride;
-    const int nvec = d / VN;
+    int nvec = d / VN;
+    if (source_rows > 0 && (row < 0 || row >= source_rows)) {   // outside the caller's buffer: never read, scored as zeros
+        if (lane == 0) atomicOr(d_status, ARROL_DEV_BAD_INDEX);
+        nvec = 0;
+    }
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     // eight independent 16-byte loads of x (and of w) in flight per lane: a 4 KB row is one round trip
     for (int c0 = lane; c0 < nvec; c0 += 256) {
@@ -112,7 +117,8 @@ __global__ void __launch_bounds__(MLP_THREADS)
 score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index,
                       int N, int d, int h, const T* __restrict__ W1, const T* __restrict__ b1,
                       const T* __restrict__ w2, float* __restrict__ partial,
-                      float* __restrict__ u_out /* [N][h] pre-activations, or NULL */, int k_len) {
+                      float* __restrict__ u_out /* [N][h] pre-activations, or NULL */, int k_len,
+                      int64_t source_rows, uint32_t* d_status) {
     constexpr int VN = Vec16<T>::N;
     constexpr int VPR = TK / VN;                       // 16-byte vectors per tile row per K chunk
     constexpr int NV = TM * VPR / MLP_THREADS;         // vectors per thread per operand per chunk (2 or 4)
@@ -136,7 +142,11 @@ score_mlp_tile_kernel(const T* __restrict__ hidden, int64_t row_stride, const in
         const int m = m0 + rr[i], j = j0 + rr[i];
         xrow[i] = nullptr;
         wrow[i] = nullptr;
-        if (m < N) xrow[i] = hidden + (row_index ? row_index[m] : (int64_t)m) * row_stride;
+        if (m < N) {
+            const int64_t row = row_index ? row_index[m] : (int64_t)m;
+            if (source_rows > 0 && (row < 0 || row >= source_rows)) atomicOr(d_status, ARROL_DEV_BAD_INDEX);   // read as zeros
+            else xrow[i] = hidden + row * row_stride;
+        }
         if (j < h) wrow[i] = W1 + (int64_t)j * d;
     }
     const int k_end = SPLITK ? min(d, ((int)blockIdx.z + 1) * k_len) : d;
@@ -288,7 +298,8 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
         const int blocks = (N + warps_per_block - 1) / warps_per_block;
         ARROL_CUDA_OK(arrol_launch_pdl(score_linear_kernel<T>, dim3(blocks), dim3(32 * warps_per_block), 0, s, hid,
                                        row_stride, row_index, N, head->d, static_cast<const T*>(head->W1),
-                                       static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q));
+                                       static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q,
+                                       ctx->source_rows, ctx->d_status));
         ctx->launches += 1;
     } else {
         if constexpr (sizeof(T) == 2) {
@@ -311,7 +322,7 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
             dim3 grid(m_tiles, h_tiles, splits);
             score_mlp_tile_kernel<T, true><<<grid, MLP_THREADS, 0, s>>>(
                 hid, row_stride, row_index, N, head->d, head->h, static_cast<const T*>(head->W1), nullptr, nullptr,
-                ctx->d_scratch, nullptr, k_len);
+                ctx->d_scratch, nullptr, k_len, ctx->source_rows, ctx->d_status);
             score_mlp_splitk_finish_kernel<T><<<(N + 3) / 4, 128, 0, s>>>(
                 ctx->d_scratch, splits, N, head->h, static_cast<const T*>(head->b1), static_cast<const T*>(head->w2),
                 static_cast<const T*>(head->b2), B, q_lut, score, prob, bin, q);
@@ -319,7 +330,8 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
             dim3 grid(m_tiles, h_tiles);
             score_mlp_tile_kernel<T, false><<<grid, MLP_THREADS, 0, s>>>(
                 hid, row_stride, row_index, N, head->d, head->h, static_cast<const T*>(head->W1),
-                static_cast<const T*>(head->b1), static_cast<const T*>(head->w2), ctx->d_scratch, nullptr, 0);
+                static_cast<const T*>(head->b1), static_cast<const T*>(head->w2), ctx->d_scratch, nullptr, 0,
+                ctx->source_rows, ctx->d_status);
             score_mlp_finish_kernel<T><<<(N + 255) / 256, 256, 0, s>>>(ctx->d_scratch, N, h_tiles,
                                                                       static_cast<const T*>(head->b2), B, q_lut,
                                                                       score, prob, bin, q);
@@ -341,12 +353,12 @@ int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_str
         score_mlp_tile_kernel<float, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const float*>(hidden), row_stride, row_index, N, head->d, head->h,
             static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
-            static_cast<const float*>(head->w2), partial, u_out, 0);
+            static_cast<const float*>(head->w2), partial, u_out, 0, ctx->source_rows, ctx->d_status);
     else
         score_mlp_tile_kernel<__nv_bfloat16, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const __nv_bfloat16*>(hidden), row_stride, row_index, N, head->d, head->h,
             static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
-            static_cast<const __nv_bfloat16*>(head->w2), partial, u_out, 0);
+            static_cast<const __nv_bfloat16*>(head->w2), partial, u_out, 0, ctx->source_rows, ctx->d_status);
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     return ARROL_OK;
@@ -450,14 +462,14 @@ extern "C" int arrol_score_partial_static(const void* hidden, int64_t row_stride
         score_mlp_tile_kernel<float, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const float*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const float*>(head->W1), static_cast<const float*>(head->b1),
-            static_cast<const float*>(head->w2), partial, nullptr, 0);
+            static_cast<const float*>(head->w2), partial, nullptr, 0, (int64_t)0, nullptr);
         score_mlp_finish_kernel<float><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const float*>(head->b2), B, q_lut, score, prob, bin, q);
     } else {
         score_mlp_tile_kernel<__nv_bfloat16, false><<<grid, MLP_THREADS, 0, s>>>(
             static_cast<const __nv_bfloat16*>(hidden), row_stride_elems, row_index, N, head->d, head->h,
             static_cast<const __nv_bfloat16*>(head->W1), static_cast<const __nv_bfloat16*>(head->b1),
-            static_cast<const __nv_bfloat16*>(head->w2), partial, nullptr, 0);
+            static_cast<const __nv_bfloat16*>(head->w2), partial, nullptr, 0, (int64_t)0, nullptr);
         score_mlp_finish_kernel<__nv_bfloat16><<<(N + 255) / 256, 256, 0, s>>>(
             partial, N, h_tiles, static_cast<const __nv_bfloat16*>(head->b2), B, q_lut, score, prob, bin, q);
     }

@@ -36,16 +36,22 @@ constexpr size_t S_SMEM_BYTES = (size_t)S_STAGES * S_STAGE_BYTES + 1024 + S_TAIL
 // one warp per rollout: 16-byte copies, all of a row's loads in flight before the first store
 __global__ void __launch_bounds__(128)
 pack_rows_kernel(const __nv_bfloat16* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index,
-                 int N, int d, __nv_bfloat16* __restrict__ out) {
+                 int N, int d, __nv_bfloat16* __restrict__ out, int64_t source_rows, uint32_t* d_status) {
     pdl_launch_dependents();
     pdl_wait();
     hidden = pdl_acquire(hidden); row_index = pdl_acquire(row_index);
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (i >= N) return;
-    const uint4* src = reinterpret_cast<const uint4*>(hidden + row_index[i] * row_stride);
+    const int64_t row = row_index[i];
+    const uint4* src = reinterpret_cast<const uint4*>(hidden + row * row_stride);
     uint4* dst = reinterpret_cast<uint4*>(out + (int64_t)i * d);
     const int nvec = d / 8;
+    if (source_rows > 0 && (row < 0 || row >= source_rows)) {   // outside the caller's buffer: never read, packed as zeros
+        if (lane == 0) atomicOr(d_status, ARROL_DEV_BAD_INDEX);
+        for (int c = lane; c < nvec; c += 32) dst[c] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
     for (int c0 = lane; c0 < nvec; c0 += 256) {
         uint4 v[8];
 #pragma unroll
@@ -264,7 +270,7 @@ int arrol_internal_score_mlp_tc(arrol_ctx* ctx, const void* hidden, int64_t row_
     if (row_index) {
         ARROL_CUDA_OK(arrol_launch_pdl(pack_rows_kernel, dim3((N + 3) / 4), dim3(128), 0, s,
                                        static_cast<const __nv_bfloat16*>(hidden), row_stride, row_index, N, d,
-                                       static_cast<__nv_bfloat16*>(ctx->d_pack)));
+                                       static_cast<__nv_bfloat16*>(ctx->d_pack), ctx->source_rows, ctx->d_status));
         ctx->launches += 1;
         x = ctx->d_pack;
         ld = d;

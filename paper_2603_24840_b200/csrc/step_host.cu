@@ -1,25 +1,28 @@
 // arrol_prune_rebatch_host: one whole prune-and-rebatch step for callers whose per-step data is in host memory
 // (Algorithm 1, frontend: filter pruned rollouts, re-batch, log-probs on the survivors).
 //
-// Only what the step needs crosses the bus: the N hidden rows at the detection length (for the head), the small
-// per-rollout arrays and token ids, and then -- once the keep mask is known -- the survivors' hidden rows, which are
-// copied straight into their packed positions (the copy engine does the row compaction).  Those uploads run on a
+// Only what the step needs crosses the bus: the N hidden rows at the detection length (for the head; packed into a
+// pinned staging block on the host and sent as one copy), the small per-rollout arrays, and then -- once the keep
+// mask is known -- the survivors' hidden rows and token ids, which are copied straight into their packed positions
+// (the copy engine does the compaction).  Those uploads run on a
 // second stream in token chunks, and the log-prob kernel of chunk c starts as soon as chunk c has landed, so the
 // upload of the survivors is hidden behind the tensor-core work.  One host synchronisation in the middle (the mask
 // must reach the host to plan the copies) and one at the end.
+#include <cstring>
 #include <vector>
 
 #include "arrol_internal.h"
 
 namespace {
 
-__global__ void row_index_kernel(const int64_t* __restrict__ src_tok_off, int N, int cutoff,
-                                 int64_t* __restrict__ row_index) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < N) row_index[i] = src_tok_off[i] + (int64_t)(cutoff - 1);
-}
-
 constexpr int64_t CHUNK_TOKENS = 2 * 74 * 128;   // token tiles per chunk = a multiple of the SM count
+
+// tokens per log-prob launch when T tokens are uploaded: whole multiples of CHUNK_TOKENS, at most one event per chunk
+int64_t chunk_for(int64_t T) {
+    int64_t chunk = CHUNK_TOKENS;
+    while ((T + chunk - 1) / chunk > ARROL_COPY_EVENTS) chunk += CHUNK_TOKENS;
+    return chunk < T ? chunk : (T > 0 ? T : 1);
+}
 
 }  // namespace
 
@@ -28,7 +31,8 @@ extern "C" int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* s
     if (st->P < 0 || st->G < 1 || st->K < 1 || st->K > st->G || st->cutoff < 1 || st->d <= 0 || st->V <= 0 ||
         st->T_src < 0 || st->dst_capacity_tokens < 0)
         return ARROL_ERR_INVALID_ARG;
-    if (st->head.dtype != ARROL_BF16) return ARROL_ERR_UNSUPPORTED;
+    if (st->head.dtype != ARROL_BF16 || st->d % 8 != 0) return ARROL_ERR_UNSUPPORTED;
+    if (st->head.d != st->d) return ARROL_ERR_INVALID_ARG;      // the head reads whole hidden rows
     const int64_t N64 = (int64_t)st->P * st->G;
     if (N64 > ARROL_MAX_HOST_N) return ARROL_ERR_UNSUPPORTED;
     const int N = (int)N64;
@@ -37,13 +41,17 @@ extern "C" int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* s
         return ARROL_OK;
     }
     const void* need[] = {st->h_hidden, st->h_src_tokens, st->h_lengths, st->h_src_tok_off, st->h_rewards,
-                          st->W_vocab, st->d_hidden, st->d_src_tokens, st->d_lengths, st->d_src_tok_off,
-                          st->d_row_index, st->d_rewards, st->d_score, st->d_prob, st->d_q, st->d_keep,
+                          st->W_vocab, st->d_hidden, st->d_lengths, st->d_src_tok_off,
+                          st->d_rewards, st->d_score, st->d_prob, st->d_q, st->d_keep,
                           st->d_survivor_idx, st->d_cu_seqlens, st->d_adv, st->d_num, st->d_dst_tokens,
                           st->d_dst_rows, st->d_logp, st->d_workspace, st->h_logp, st->h_adv, st->h_cu_seqlens,
                           st->h_survivor_idx, st->h_num};
     for (const void* p : need)
         if (!p) return ARROL_ERR_INVALID_ARG;
+    // the workspace must serve the largest chunk any T <= capacity can lead to (its size is monotone in the tokens)
+    if (!arrol_aligned(st->d_workspace, 256) ||
+        arrol_token_logprob_workspace(ctx, chunk_for(st->dst_capacity_tokens), st->d, st->V) > st->workspace_bytes)
+        return ARROL_ERR_WORKSPACE;
     for (int i = 0; i < N; ++i) {
         const int64_t row = st->h_src_tok_off[i] + st->cutoff - 1;
         if (st->h_src_tok_off[i] < 0 || row >= st->T_src || st->h_lengths[i] < 0 ||
@@ -63,16 +71,19 @@ extern "C" int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* s
     ARROL_CUDA_OK(cudaMemcpyAsync(st->d_lengths, st->h_lengths, sizeof(int32_t) * N, cudaMemcpyHostToDevice, s));
     ARROL_CUDA_OK(cudaMemcpyAsync(st->d_src_tok_off, st->h_src_tok_off, sizeof(int64_t) * N, cudaMemcpyHostToDevice, s));
     ARROL_CUDA_OK(cudaMemcpyAsync(st->d_rewards, st->h_rewards, sizeof(float) * N, cudaMemcpyHostToDevice, s));
-    ARROL_CUDA_OK(cudaMemcpyAsync(st->d_src_tokens, st->h_src_tokens, sizeof(int32_t) * (size_t)st->T_src,
-                                  cudaMemcpyHostToDevice, s));
-    for (int i = 0; i < N; ++i) {   // the hidden row of every rollout at the detection length, at its own place
-        const size_t off = (size_t)(st->h_src_tok_off[i] + st->cutoff - 1) * rb;
-        ARROL_CUDA_OK(cudaMemcpyAsync(d_hidden + off, h_hidden + off, rb, cudaMemcpyHostToDevice, s));
+    // the hidden row of every rollout at the detection length, packed as [N, d] at the start of d_hidden: through
+    // the pinned staging block as one copy when it fits, else row by row
+    if ((size_t)N * rb <= ARROL_STAGE_BYTES) {
+        for (int i = 0; i < N; ++i)
+            std::memcpy(ctx->h_stage + (size_t)i * rb, h_hidden + (size_t)(st->h_src_tok_off[i] + st->cutoff - 1) * rb, rb);
+        ARROL_CUDA_OK(cudaMemcpyAsync(d_hidden, ctx->h_stage, (size_t)N * rb, cudaMemcpyHostToDevice, s));
+    } else {
+        for (int i = 0; i < N; ++i)
+            ARROL_CUDA_OK(cudaMemcpyAsync(d_hidden + (size_t)i * rb,
+                                          h_hidden + (size_t)(st->h_src_tok_off[i] + st->cutoff - 1) * rb, rb,
+                                          cudaMemcpyHostToDevice, s));
     }
-    row_index_kernel<<<(N + 255) / 256, 256, 0, s>>>(st->d_src_tok_off, N, st->cutoff, st->d_row_index);
-    ARROL_CUDA_OK(cudaGetLastError());
-    ctx->launches += 1;
-    int rc = arrol_score_partial(ctx, st->d_hidden, st->d, st->d_row_index, N, &st->head, &st->calib, st->d_score,
+    int rc = arrol_score_partial(ctx, st->d_hidden, st->d, nullptr, N, &st->head, &st->calib, st->d_score,
                                  st->d_prob, nullptr, st->d_q, stream);
     if (rc != ARROL_OK) return rc;
     rc = arrol_select(ctx, st->d_q, st->P, st->G, st->K, st->rho, 0, st->d_keep, stream);
@@ -91,23 +102,24 @@ extern "C" int arrol_prune_rebatch_host(arrol_ctx* ctx, const arrol_host_step* s
         }
     const int64_t T = cu.back();
 
-    // scan, advantages and token ids on the device (no row payload: the rows arrive packed)
-    rc = arrol_compact(ctx, st->d_keep, st->d_lengths, st->d_src_tok_off, N, st->G, st->d_src_tokens, nullptr, 0,
-                       st->d_rewards, st->eps, st->ddof, st->dst_capacity_tokens, st->d_dst_tokens, nullptr,
+    // scan and advantages on the device (no per-token payload: rows and token ids arrive packed)
+    rc = arrol_compact(ctx, st->d_keep, st->d_lengths, st->d_src_tok_off, N, st->G, nullptr, nullptr, 0,
+                       st->d_rewards, st->eps, st->ddof, st->dst_capacity_tokens, nullptr, nullptr,
                        st->d_cu_seqlens, st->d_survivor_idx, st->d_adv, nullptr, nullptr, st->d_num, stream);
     if (rc != ARROL_OK) return rc;
 
     if (T > 0 && T <= st->dst_capacity_tokens) {
-        int64_t chunk = CHUNK_TOKENS;
-        while ((T + chunk - 1) / chunk > ARROL_COPY_EVENTS) chunk += CHUNK_TOKENS;
-        if (arrol_token_logprob_workspace(ctx, chunk < T ? chunk : T, st->d, st->V) > st->workspace_bytes) chunk = T;
+        const int64_t chunk = chunk_for(T);
         int64_t c = 0;                       // next chunk to launch: tokens [c*chunk, min(T, (c+1)*chunk))
         for (size_t k = 0; k < surv.size(); ++k) {
             const int64_t len = cu[k + 1] - cu[k];
-            if (len > 0)
+            if (len > 0) {
                 ARROL_CUDA_OK(cudaMemcpyAsync(d_dst_rows + (size_t)cu[k] * rb,
                                               h_hidden + (size_t)st->h_src_tok_off[surv[k]] * rb, (size_t)len * rb,
                                               cudaMemcpyHostToDevice, ctx->copy_stream));
+                ARROL_CUDA_OK(cudaMemcpyAsync(st->d_dst_tokens + cu[k], st->h_src_tokens + st->h_src_tok_off[surv[k]],
+                                              (size_t)len * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->copy_stream));
+            }
             const bool last = (k + 1 == surv.size());
             while (c * chunk < T && (cu[k + 1] >= (c + 1) * chunk || last)) {
                 const int64_t t0 = c * chunk, t1 = (t0 + chunk < T) ? t0 + chunk : T;

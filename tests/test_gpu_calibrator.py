@@ -150,3 +150,31 @@ def test_calibrated_loop_feeds_scoring_and_compaction(ctx):
     assert np.abs(outs["adv"].cpu().numpy()[:S] - adv_ref).max() <= 1e-5
     counts = keep_ref.reshape(P, G).sum(1)
     assert counts.min() < counts.max()                                   # ragged groups were exercised
+
+
+def test_update_with_another_shape_leaves_the_state_untouched(ctx):
+    """The state was initialised with (B, cap); an update that names another pair, or a state that was never
+    initialised, is reported through the status word and changes nothing."""
+    cal = CAL.Calibrator(ctx, 128, 256)
+    sp = CAL.survival()
+    bins = torch.arange(50, dtype=torch.int32, device="cuda")
+    rew = (torch.arange(50, device="cuda") % 2).float()
+    cal.update(bins, rew, sp)
+    torch.cuda.synchronize()
+    good = cal.state.clone()
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
+    for n_bins, cap in ((64, 256), (128, 512)):
+        B._check(CAL._lib().arrol_calib_update(ctx.handle, B._ptr(cal.state), n_bins, cap, B._ptr(bins), B._ptr(rew),
+                                               None, 50, CAL.C.byref(sp), B._stream()), "arrol_calib_update")
+        torch.cuda.synchronize()
+        assert B.arrol_poll_status(ctx, raise_on_error=False) == 8          # ARROL_DEV_BAD_STATE
+        assert torch.equal(cal.state, good)
+    raw = torch.zeros(CAL.arrol_calib_state_bytes(128, 256), dtype=torch.uint8, device="cuda")   # never initialised
+    B._check(CAL._lib().arrol_calib_update(ctx.handle, B._ptr(raw), 128, 256, B._ptr(bins), B._ptr(rew), None, 50,
+                                           CAL.C.byref(sp), B._stream()), "arrol_calib_update")
+    torch.cuda.synchronize()
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 8
+    assert not raw.any()
+    cal.update(bins, rew, sp)                                                # the right pair still works
+    torch.cuda.synchronize()
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0

@@ -13,7 +13,8 @@ from paper_2603_24840_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("T,d,V", [(130, 64, 300), (300, 192, 1000), (2000, 128, 4096), (140, 256, 20000), (19200, 64, 512)])
+@pytest.mark.parametrize("T,d,V", [(130, 64, 300), (300, 192, 1000), (2000, 128, 4096), (140, 256, 20000), (19200, 64, 512),
+                                   (200, 128, 151936)])
 def test_token_confidence_and_logprob_from_one_launch(T, d, V):
     ctx = B.Context(0)
     g = np.random.default_rng(T + V)
@@ -47,7 +48,7 @@ def test_trace_confidence_matches_oracle():
     S, T = len(ell), int(cu[-1])
     Hs = (g.random(T) * 1e5 + 1e6).astype(np.float32)
     d_num = torch.tensor([S, T], dtype=torch.int64, device="cuda")
-    for mode, window in ((0, 1), (1, 1), (1, 16), (1, 2048), (1, 100000)):
+    for mode, window in ((0, 1), (1, 1), (1, 16), (1, 2048), (1, 100000), (2, 1), (2, 16), (2, 2048), (2, 100000)):
         ref = oc.trace_confidence(Hs.astype(np.float64), cu, window=window, mode=mode)
         out = torch.full((S,), -1.0, device="cuda")
         CF.arrol_trace_confidence(ctx, torch.from_numpy(Hs).cuda(), torch.from_numpy(cu).cuda(), d_num, S, out,
@@ -55,6 +56,47 @@ def test_trace_confidence_matches_oracle():
         torch.cuda.synchronize()
         assert np.abs(out.cpu().numpy() - ref).max() <= 1e-6 * np.abs(ref).max()
     with pytest.raises(B.ArrolError) as e:
-        CF.arrol_trace_confidence(ctx, out, out, d_num, S, out, mode=2)
+        CF.arrol_trace_confidence(ctx, out, out, d_num, S, out, mode=3)
     assert e.value.code == -2
+    ctx.close()
+
+
+def test_bottom_tenth_on_long_and_tied_traces():
+    """mode 2 beyond the shared-memory prefix (len > 8192) and on values with many exact ties."""
+    ctx = B.Context(0)
+    g = np.random.default_rng(5)
+    ell = np.array([8192, 8193, 20000, 3000, 77])
+    cu = np.concatenate([[0], np.cumsum(ell)]).astype(np.int64)
+    S, T = len(ell), int(cu[-1])
+    Hs = g.integers(0, 4, size=T).astype(np.float32) * 1000.0          # four distinct values: ties everywhere
+    Hs[cu[3]:cu[4]] = -g.random(3000).astype(np.float32)                # a negative trace: the key map handles the sign
+    d_num = torch.tensor([S, T], dtype=torch.int64, device="cuda")
+    for window in (1, 7, 4096):
+        ref = oc.trace_confidence(Hs.astype(np.float64), cu, window=window, mode=2)
+        out = torch.full((S,), -1.0, device="cuda")
+        CF.arrol_trace_confidence(ctx, torch.from_numpy(Hs).cuda(), torch.from_numpy(cu).cuda(), d_num, S, out,
+                                  window=window, mode=2)
+        torch.cuda.synchronize()
+        assert np.abs(out.cpu().numpy() - ref).max() <= 1e-6 * max(np.abs(ref).max(), 1.0)
+    ctx.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_trace_count_beyond_the_arrays_is_clamped(mode):
+    """d_num[0] larger than S_max: only S_max traces are reduced and nothing past trace_conf[S_max] is written."""
+    ctx = B.Context(0)
+    g = np.random.default_rng(6)
+    ell = g.integers(1, 300, size=12)
+    cu = np.concatenate([[0], np.cumsum(ell)]).astype(np.int64)
+    S_max, T = len(ell), int(cu[-1])
+    Hs = g.random(T).astype(np.float32) * 50
+    d_num = torch.tensor([S_max + 1000, T], dtype=torch.int64, device="cuda")     # a stale / oversized count
+    out = torch.full((S_max + 64,), -7.0, device="cuda")                          # canaries after the S_max results
+    CF.arrol_trace_confidence(ctx, torch.from_numpy(Hs).cuda(), torch.from_numpy(cu).cuda(), d_num, S_max, out,
+                              window=16, mode=mode)
+    torch.cuda.synchronize()
+    ref = oc.trace_confidence(Hs.astype(np.float64), cu, window=16, mode=mode)
+    got = out.cpu().numpy()
+    assert np.abs(got[:S_max] - ref).max() <= 1e-6 * np.abs(ref).max()
+    assert np.all(got[S_max:] == -7.0)
     ctx.close()

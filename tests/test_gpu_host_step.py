@@ -22,8 +22,8 @@ def _host_step(pr, w):
          "h_survivor_idx": torch.empty(N, dtype=torch.int32).pin_memory(),
          "h_num": torch.empty(2, dtype=torch.int64).pin_memory()}
     z = lambda t: torch.zeros_like(t)
-    dv = {"W_vocab": pr.W_vocab, "d_hidden": z(pr.src_rows), "d_src_tokens": z(pr.src_tokens), "d_lengths": z(pr.lengths),
-          "d_src_tok_off": z(pr.src_tok_off), "d_row_index": z(pr.row_index), "d_rewards": z(pr.rewards),
+    dv = {"W_vocab": pr.W_vocab, "d_hidden": torch.zeros((N, w.d), dtype=torch.bfloat16, device="cuda"),
+          "d_lengths": z(pr.lengths), "d_src_tok_off": z(pr.src_tok_off), "d_rewards": z(pr.rewards),
           "d_score": z(pr.score), "d_prob": z(pr.prob), "d_q": z(pr.q), "d_keep": z(pr.keep),
           "d_survivor_idx": z(pr.survivor_idx), "d_cu_seqlens": z(pr.cu_seqlens), "d_adv": z(pr.adv),
           "d_num": z(pr.d_num), "d_dst_tokens": z(pr.dst_tokens), "d_dst_rows": z(pr.dst_rows), "d_logp": z(pr.logp),
@@ -64,4 +64,27 @@ def test_host_step_matches_device_path_and_oracle(name):
                                      pr.dst_tokens.cpu().numpy()[rows])
     assert np.abs(h["h_logp"].numpy()[rows] - lp_ref).max() <= 2e-3
     assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+    pr.ctx.close()
+
+
+def test_host_step_validates_before_it_copies():
+    """A head of another width, a hidden width that is no multiple of 8 and a short workspace are refused up front."""
+    w = synth.WORKLOADS["mini"]
+    pr = PruneRebatch(w, inputs=host_inputs(w))
+    h, dv, (head, tensors) = _host_step(pr, w)
+    scal = dict(P=w.P, G=w.G, K=w.K, cutoff=w.cutoff, d=w.d, V=w.V, ddof=0, rho=w.rho, eps=1e-6, inv_temperature=1.0,
+                T_src=pr.T_src, dst_capacity_tokens=pr.cap)
+    dv["d_lengths"].fill_(-3)
+    step = B.make_host_step(scal, head, pr.q_lut, tensors)
+    step.head.d = w.d - 8
+    with pytest.raises(B.ArrolError) as e:
+        B.arrol_prune_rebatch_host(pr.ctx, step)
+    assert e.value.code == -1
+    step = B.make_host_step(scal, head, pr.q_lut, tensors)
+    step.workspace_bytes = 16
+    with pytest.raises(B.ArrolError) as e:
+        B.arrol_prune_rebatch_host(pr.ctx, step)
+    assert e.value.code == -3
+    torch.cuda.synchronize()
+    assert torch.all(dv["d_lengths"] == -3)            # nothing was uploaded by the refused calls
     pr.ctx.close()

@@ -2,15 +2,20 @@
 (frozen memory plans, host applications that own the device heap, latency-critical loops).  It keeps its scratch
 in a fixed array inside the library, takes no context and allocates nothing.
 
-Checked here through the C ABI against the regular entry point arrol_score_partial on the same inputs, twice in a
-row with different shapes, so that whatever the first call leaves in the shared scratch cannot leak into the
-second.  This file sorts last on purpose: a run that stops at the first failure has already run everything else.
+Checked here through the C ABI against the regular entry point arrol_score_partial and against the CPU oracle on
+the same inputs, three calls in a row with different shapes, so that whatever one call leaves in the shared scratch
+cannot leak into the next.  The two entry points run different kernels for a bf16 head (the regular one contracts
+on the tensor cores, this one in fp32 on the ordinary ALUs), so scores agree within the scoring tolerance, a bin may
+differ by one only next to a bin edge, and q is always the table entry of the call's own bin.
+This file sorts last on purpose: a run that stops at the first failure has already run everything else.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2603_24840_b200 import binding as B
+from paper_2603_24840_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
@@ -46,8 +51,25 @@ def test_static_entry_matches_the_regular_entry_on_two_calls_in_a_row():
             torch.cuda.synchronize()
             assert (s0 - s1).abs().max().item() <= PROB_TOL
             assert (p0 - p1).abs().max().item() <= PROB_TOL
-            assert torch.equal(b0, b1) and torch.equal(q0, q1)      # same kernels: the table look-up agrees exactly
             assert not torch.any(p1 == 7.0)
+            # against the fp64 oracle: scores and probabilities within the scoring tolerance
+            oa = synth.as_oracle_array
+            s_ref = oracle.head_score(oa(x), oa(head["W1"]), oa(head["b1"]), oa(head["w2"]), oa(head["b2"]),
+                                      row_index=ridx.cpu().numpy(), h=h)
+            lut_h = lut.cpu().numpy()
+            p_ref, b_ref, _ = oracle.prob_map(s_ref, lut_h)
+            assert np.abs(s1.cpu().numpy() - s_ref).max() <= PROB_TOL
+            assert np.abs(p1.cpu().numpy() - p_ref).max() <= PROB_TOL
+            # bins: the oracle's bin, or its neighbour where 128 s' lies within the tolerance of a bin edge;
+            # q is bit-equal to the table entry of the bin this call chose
+            bins = b1.cpu().numpy()
+            near_edge = np.abs(128 * p_ref - np.rint(128 * p_ref)) <= 128 * PROB_TOL
+            assert np.all((bins == b_ref) | (near_edge & (np.abs(bins - b_ref) <= 1)))
+            assert np.array_equal(q1.cpu().numpy(), lut_h[bins])
+            assert np.array_equal(bins, np.array([oracle.bin_index(float(v), 128) for v in p1.cpu().numpy()]))
+            same = b0 == b1
+            assert torch.equal(q0[same], q1[same])
+            assert np.all(near_edge[(~same).cpu().numpy()])          # the two entry points differ only next to an edge
     finally:
         ctx.close()
 
