@@ -618,9 +618,9 @@ def run_e2e(args, w, pr, B, torch, world, barrier):
         "h_num": torch.empty(2, dtype=torch.int64).pin_memory(),
     }
     dv = {
-        "W_vocab": pr.W_vocab, "d_hidden": torch.empty_like(pr.src_rows), "d_src_tokens": torch.empty_like(pr.src_tokens),
+        "W_vocab": pr.W_vocab, "d_hidden": torch.empty((N, w.d), dtype=torch.bfloat16, device=pr.dev),
         "d_lengths": torch.empty_like(pr.lengths), "d_src_tok_off": torch.empty_like(pr.src_tok_off),
-        "d_row_index": torch.empty_like(pr.row_index), "d_rewards": torch.empty_like(pr.rewards),
+        "d_rewards": torch.empty_like(pr.rewards),
         "d_score": pr.score, "d_prob": pr.prob, "d_q": pr.q, "d_keep": pr.keep, "d_survivor_idx": pr.survivor_idx,
         "d_cu_seqlens": pr.cu_seqlens, "d_adv": pr.adv, "d_num": pr.d_num, "d_dst_tokens": pr.dst_tokens,
         "d_dst_rows": pr.dst_rows, "d_logp": pr.logp, "d_workspace": pr.workspace,
@@ -633,12 +633,13 @@ def run_e2e(args, w, pr, B, torch, world, barrier):
     tensors = dict(h)
     tensors.update(dv)
     step = B.make_host_step(scal, head, pr.q_lut, tensors)
-    # bytes the call moves per step: small arrays and token ids, the N hidden rows at the detection length, then only
-    # the survivors' hidden rows (uploaded straight into their packed positions); results: logp[T] + per-rollout arrays
+    # bytes the call moves per step: the small per-rollout arrays, the N hidden rows at the detection length, then only
+    # the survivors' hidden rows and token ids (uploaded straight into their packed positions); results: logp[T] +
+    # per-rollout arrays
     _, T_now = pr.counts()
     row_bytes = w.d * 2
-    h2d = sum(h[k].numel() * h[k].element_size() for k in ("h_src_tokens", "h_lengths", "h_src_tok_off", "h_rewards"))
-    h2d += (N + T_now) * row_bytes
+    h2d = sum(h[k].numel() * h[k].element_size() for k in ("h_lengths", "h_src_tok_off", "h_rewards"))
+    h2d += (N + T_now) * row_bytes + 4 * T_now
     d2h = sum(h[k].numel() * h[k].element_size() for k in ("h_adv", "h_cu_seqlens", "h_survivor_idx", "h_num")) + 4 * T_now + N
     n_e2e = max(1, min(args.steps, 5))
     for _ in range(2):

@@ -161,6 +161,29 @@ int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab,
                         int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                         float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- Selected-token log-probability straight from the pre-prune buffer (Section 4.3 (ii): the frontend "filters
+ * out pruned rollouts and re-batches the surviving ones to compute log-probabilities"; Algorithm 1) -------------
+ * arrol_token_logprob on the survivors WITHOUT a packed copy of their hidden rows: packed token t of survivor s
+ * (cu_seqlens[s] <= t < cu_seqlens[s+1]) is row src_tok_off[survivor_idx[s]] + (t - cu_seqlens[s]) of src_rows, and
+ * the kernel's loads follow that mapping, so arrol_compact can be called without the hidden-row plane
+ * (src_rows = dst_rows = NULL) and [T, d] never exists in memory.
+ *   src_rows [source_rows, d] bf16 row-major, 16-byte aligned; source_rows <= 2^31 - 129;
+ *   cu_seqlens [>= S_max + 1] int64, survivor_idx [>= S_max] int32, d_num [2] int64 = {S, T}: the outputs of
+ *   arrol_compact (S is clamped to S_max, T to T_max);  src_tok_off [N] int64: the array given to arrol_compact;
+ *   targets [T_max] int32 in packed order (arrol_compact's dst_tokens);  logp, lse, d, V, inv_temperature as in
+ *   arrol_token_logprob.  workspace: arrol_token_logprob_gathered_workspace(ctx, S_max, T_max, d, V) bytes, 256-byte
+ *   aligned: the split records of arrol_token_logprob plus S_max * 128 * d * 2 bytes, into which a first small
+ *   kernel copies the token tiles that cross a survivor boundary (at most one per survivor); every other tile is
+ *   read in place.
+ * Results equal arrol_token_logprob on the packed rows bit for bit.  Source rows are trusted to lie inside
+ * [0, source_rows) (see arrol_set_source_rows for arrol_compact's check of the same offsets). */
+size_t arrol_token_logprob_gathered_workspace(arrol_ctx* ctx, int32_t S_max, int64_t T_max, int32_t d, int32_t V);
+int arrol_token_logprob_gathered(arrol_ctx* ctx, const void* src_rows, int64_t source_rows, const void* W_vocab,
+                                 const int32_t* targets, const int64_t* cu_seqlens, const int32_t* survivor_idx,
+                                 const int64_t* src_tok_off, const int64_t* d_num, int32_t S_max, int64_t T_max,
+                                 int32_t d, int32_t V, float inv_temperature, float* logp, float* lse,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- Prune step in one call (Algorithm 1: quality check at the detection length, filter, re-batch) ----------
  * arrol_score_partial -> arrol_select -> arrol_compact issued back to back on `stream` with N = P * G; every field
  * has the meaning, layout and nullability of the argument of the same name in those calls.  Asynchronous.
@@ -429,9 +452,17 @@ int64_t arrol_launch_count(arrol_ctx* ctx);
  *   ARROL_HOOK_SPIN_LIMIT            value = tries per wait (0 restores the normal limit of 2^26)
  *   ARROL_HOOK_MUTE_LOGPROB_PRODUCER value != 0: the kernel's producer issues no copies, so the other roles' waits
  *                                    run out after the limit above; outputs of such a call are not written.
+ *   ARROL_HOOK_LOGPROB_TIMING_BUFFER value = device address of a buffer of 4 x uint64 per work item (0 = off), and
+ *   ARROL_HOOK_LOGPROB_TIMING_ITEMS  value = its capacity in work items: while set, every work item (token tile x
+ *                                    vocabulary split) i < capacity of an arrol_token_logprob launch records
+ *                                    {globaltimer at start, globaltimer at end, SM clock at start, SM clock at end}
+ *                                    of its epilogue, from which a benchmark derives the SM clock the kernel ran at
+ *                                    (cycles / nanoseconds) without reading or setting any GPU clock control.
  * Returns INVALID_ARG for an unknown key or a limit outside [0, 2^26]. */
 #define ARROL_HOOK_SPIN_LIMIT 1
 #define ARROL_HOOK_MUTE_LOGPROB_PRODUCER 2
+#define ARROL_HOOK_LOGPROB_TIMING_BUFFER 3
+#define ARROL_HOOK_LOGPROB_TIMING_ITEMS 4
 int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value);
 
 #ifdef __cplusplus

@@ -27,6 +27,7 @@ EXPORTS = [
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
     "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
     "arrol_prune_step", "arrol_token_logprob_splits", "arrol_test_hook", "arrol_set_source_rows",
+    "arrol_token_logprob_gathered", "arrol_token_logprob_gathered_workspace",
 ]
 
 
@@ -108,6 +109,10 @@ def load_library():
     lib.arrol_token_logprob.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                         C.c_int32, C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_size_t, C.c_void_p]
+    lib.arrol_token_logprob_gathered.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_int32,
+                                                 C.c_int32, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                                 C.c_void_p]
     lib.arrol_prune_rebatch_host.argtypes = [C.c_void_p, C.POINTER(_HostStep), C.c_void_p]
     lib.arrol_prune_rebatch_host.restype = C.c_int
     lib.arrol_score_partial_static.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.POINTER(_Head),
@@ -273,7 +278,26 @@ def arrol_token_logprob(ctx: Context, hidden, W_vocab, targets, T_max: int, d: i
                                               _stream(stream)), "arrol_token_logprob")
 
 
-HOOK_SPIN_LIMIT, HOOK_MUTE_LOGPROB_PRODUCER = 1, 2
+def arrol_token_logprob_gathered_workspace(ctx: Context, S_max: int, T_max: int, d: int, V: int) -> int:
+    lib = load_library()
+    lib.arrol_token_logprob_gathered_workspace.restype = C.c_size_t
+    lib.arrol_token_logprob_gathered_workspace.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int32, C.c_int32]
+    return int(lib.arrol_token_logprob_gathered_workspace(ctx.handle, int(S_max), int(T_max), int(d), int(V)))
+
+
+def arrol_token_logprob_gathered(ctx: Context, src_rows, W_vocab, targets, cu_seqlens, survivor_idx, src_tok_off, d_num,
+                                 S_max: int, T_max: int, d: int, V: int, logp, workspace, lse=None,
+                                 inv_temperature: float = 1.0, source_rows: Optional[int] = None, stream=None):
+    """Log-probs of the packed survivor tokens with the hidden rows read from the pre-prune buffer `src_rows`."""
+    rows = src_rows.shape[0] if source_rows is None else int(source_rows)
+    _check(load_library().arrol_token_logprob_gathered(
+        ctx.handle, _ptr(src_rows), rows, _ptr(W_vocab), _ptr(targets), _ptr(cu_seqlens), _ptr(survivor_idx),
+        _ptr(src_tok_off), _ptr(d_num), int(S_max), int(T_max), int(d), int(V), float(inv_temperature), _ptr(logp),
+        _ptr(lse), _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+        _stream(stream)), "arrol_token_logprob_gathered")
+
+
+HOOK_SPIN_LIMIT, HOOK_MUTE_LOGPROB_PRODUCER, HOOK_LOGPROB_TIMING_BUFFER, HOOK_LOGPROB_TIMING_ITEMS = 1, 2, 3, 4
 
 
 def arrol_test_hook(ctx: Context, key: int, value: int):

@@ -52,7 +52,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
                 and os.path.getmtime(obj) > max(os.path.getmtime(src), newest_header)):
             return obj
         tmp = obj + ".%d.tmp" % os.getpid()
-        subprocess.check_call([nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", tmp])
+        subprocess.check_call([nvcc] + NVCC_FLAGS + os.environ.get("ARROL_NVCC_EXTRA", "").split() +
+                              (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", tmp])
         os.replace(tmp, obj)
         return obj
 

@@ -20,6 +20,8 @@ struct arrol_ctx {
     bool score_tc_smem_set;    // the scoring kernel's dynamic shared-memory limit has been raised on this device
     bool gather_bulk_smem_set; // likewise for the bulk-copy gather kernel
     uint32_t test_spin_limit;  // arrol_test_hook: tries per pipeline wait of the log-prob kernel, 0 = the normal limit
+    unsigned long long* logprob_timing;   // arrol_test_hook: device buffer for per-work-item time stamps of the log-prob kernel
+    int64_t logprob_timing_items;         // its capacity in work items (4 words each)
     int test_mute_producer;    // arrol_test_hook: the log-prob kernel's producer issues no copies (its waits run out)
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime
     unsigned long long launches;   // kernels launched through this context (host-side count)

@@ -48,6 +48,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->gather_bulk_smem_set = false;
     ctx->test_spin_limit = 0;
     ctx->test_mute_producer = 0;
+    ctx->logprob_timing = nullptr;
+    ctx->logprob_timing_items = 0;
     ctx->encode_tiled = nullptr;
     ctx->launches = 0;
     ctx->copy_stream = nullptr;
@@ -117,6 +119,14 @@ extern "C" int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value) {
             return ARROL_OK;
         case ARROL_HOOK_MUTE_LOGPROB_PRODUCER:
             ctx->test_mute_producer = value != 0;
+            return ARROL_OK;
+        case ARROL_HOOK_LOGPROB_TIMING_BUFFER:
+            ctx->logprob_timing = reinterpret_cast<unsigned long long*>((uintptr_t)value);
+            if (!value) ctx->logprob_timing_items = 0;
+            return ARROL_OK;
+        case ARROL_HOOK_LOGPROB_TIMING_ITEMS:
+            if (value < 0) return ARROL_ERR_INVALID_ARG;
+            ctx->logprob_timing_items = value;
             return ARROL_OK;
         default:
             return ARROL_ERR_INVALID_ARG;

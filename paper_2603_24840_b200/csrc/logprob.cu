@@ -12,6 +12,18 @@
 //               maximum and sum of 2^(z log2e - max), and the target column's logit, all in registers
 // The two accumulators let the epilogue of chunk c overlap the MMAs of chunk c + 1.
 // Every wait is bounded; when one runs out the block records ARROL_DEV_WAIT_EXPIRED, drains and returns.
+//
+// Gathered variant (arrol_token_logprob_gathered; Section 4.3 (ii): the survivors are re-batched "to compute
+// log-probabilities"): the token rows are read straight from the pre-prune source buffer, so the packed copy of the
+// hidden rows never exists.  A 128-row token tile that lies inside one survivor is 128 consecutive source rows: its
+// TMA box simply starts at that source row.  Only a tile that crosses a survivor boundary is not contiguous in the
+// source; those tiles (at most one per survivor) are first copied into a small scratch block, slot = the survivor
+// of the tile's first row, by pack_boundary_tiles_kernel, and the main kernel reads them from there through a second
+// tensor map.  Every tile therefore costs the same single box per K step.  That matters beyond the tile itself: the
+// resident blocks stream the same W_vocab chunks at about the same time and share them through L2, and a block that
+// falls behind by more than the L2 holds has to re-fetch its chunks from HBM (measured with multi-box copies for the
+// boundary tiles: +10 % cycles on those tiles spread the blocks out, HBM traffic and power rose, and the SM clock
+// fell from 1.27 to 0.8 GHz under the power cap).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -51,12 +63,38 @@ struct LogprobParams {
     uint32_t spin_limit;   // tries per pipeline wait
     int mute_producer;     // test hook: the producer issues no copies
     uint32_t* d_status;
+    // gathered variant: packed token t of survivor s is source row src_tok_off[survivor_idx[s]] + (t - cu_seqlens[s])
+    const int64_t* cu_seqlens;
+    const int32_t* survivor_idx;
+    const int64_t* src_tok_off;
+    const int64_t* d_num;  // {S, T}
+    int S_max;
+    unsigned long long* timing;   // test hook: per work item {globaltimer start, end, clock64 start, end}, or NULL
+    int64_t timing_items;
 };
 
-template <bool CONF>
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Survivor of packed token row t: the last s in [0, S) with cu_seqlens[s] <= t (this skips empty survivors).
+__device__ __forceinline__ int survivor_of_row(const int64_t* __restrict__ cu_seqlens, int S, int64_t t) {
+    int lo = 0, hi = S;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (cu_seqlens[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// GATHER: map_h covers the pre-prune source rows and map_s the scratch of pre-packed boundary tiles
+// ([S_max * 128, d], slot s at rows 128 s ...); otherwise map_h covers the packed rows and map_s is unused.
+template <bool CONF, bool GATHER>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
-                     const LogprobParams p) {
+token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_s,
+                     const __grid_constant__ CUtensorMap map_w, const LogprobParams p) {
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -88,6 +126,7 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_h) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+        if constexpr (GATHER) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_s) : "memory");
     }
     if (warp == 1) {
         tcgen05_alloc(tmem_slot, TMEM_COLS);
@@ -104,15 +143,34 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
+            int S = 0;
+            if constexpr (GATHER) {
+                const int64_t s64 = p.d_num[0];
+                S = (int)(s64 < 0 ? 0 : (s64 > (int64_t)p.S_max ? (int64_t)p.S_max : s64));
+            }
             for (int64_t item = blockIdx.x; item < items && ok && !p.mute_producer; item += gridDim.x) {
                 const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
                 const int c0 = split * p.chunks_per_split;
                 const int c1 = min(c0 + p.chunks_per_split, total_chunks);
+                // where the tile's 128 rows come from: the packed rows, a run of source rows, or a scratch slot
+                const CUtensorMap* a_map = &map_h;
+                int a_row = m_tile * BM;
+                if constexpr (GATHER) {
+                    const int64_t t0 = (int64_t)m_tile * BM;
+                    const int s0 = survivor_of_row(p.cu_seqlens, S, t0);
+                    const int64_t s_end = p.cu_seqlens[s0 + 1];
+                    if (s_end < t0 + BM && s_end < T) {     // the tile runs on into the next survivor: pre-packed
+                        a_map = &map_s;
+                        a_row = s0 * BM;
+                    } else {
+                        a_row = (int)(p.src_tok_off[p.survivor_idx[s0]] + (t0 - p.cu_seqlens[s0]));
+                    }
+                }
                 for (int c = c0; c < c1 && ok; ++c) {
                     for (int ks = 0; ks < k_steps; ++ks) {
                         if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
                         mbar_expect_tx(&full[stage], STAGE_BYTES);
-                        tma_load_2d(stage_a + (size_t)stage * A_STAGE_BYTES, &map_h, ks * BK, m_tile * BM, &full[stage]);
+                        tma_load_2d(stage_a + (size_t)stage * A_STAGE_BYTES, a_map, ks * BK, a_row, &full[stage]);
                         tma_load_2d(stage_b + (size_t)stage * B_STAGE_BYTES, &map_w, ks * BK, c * BN, &full[stage]);
                         ++issued;
                         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -185,6 +243,8 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
             const int64_t t = (int64_t)m_tile * BM + row_in_tile;
             const int y = (t < T) ? p.targets[t] : -1;
             float m2 = -INFINITY, l = 0.f, zy2 = -INFINITY, sumz = 0.f;
+            const bool stamp = p.timing != nullptr && threadIdx.x == 64 && item < p.timing_items;
+            if (stamp) { p.timing[4 * item] = global_timer_ns(); p.timing[4 * item + 2] = (unsigned long long)clock64(); }
             for (int c = c0; c < c1 && ok; ++c) {
                 ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.spin_limit);
                 ok = __all_sync(0xffffffffu, ok) != 0;     // keep the warp converged for the aligned tensor-memory loads
@@ -232,6 +292,7 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 if (lane == 0) mbar_arrive(&acc_empty[acc]);
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
+            if (stamp) { p.timing[4 * item + 1] = global_timer_ns(); p.timing[4 * item + 3] = (unsigned long long)clock64(); }
             if (ok && t < T) {
                 if (p.splits == 1) {
                     const float lse2 = m2 + log2f(l);
@@ -260,6 +321,58 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
     if (warp == 1) {
         tcgen05_fence_after();
         tcgen05_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// Gathered variant, first kernel: copies every token tile that crosses a survivor boundary into its scratch slot.
+// Block s looks at the tile that holds survivor s's last row: if that tile starts inside s (so s owns it) and runs on
+// past the end of s, its rows are copied, run by run, with 16-byte loads/stores (eight in flight per thread).
+constexpr int PACK_THREADS = 256;
+__global__ void __launch_bounds__(PACK_THREADS)
+pack_boundary_tiles_kernel(const uint4* __restrict__ src_rows, const int64_t* __restrict__ cu_seqlens,
+                           const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
+                           const int64_t* __restrict__ d_num, int S_max, int64_t T_max, int vec_per_row,
+                           uint4* __restrict__ scratch) {
+    __shared__ int64_t src_row_of[BM];
+    pdl_launch_dependents();
+    pdl_wait();
+    cu_seqlens = pdl_acquire(cu_seqlens); survivor_idx = pdl_acquire(survivor_idx); d_num = pdl_acquire(d_num);
+    src_tok_off = pdl_acquire(src_tok_off); src_rows = pdl_acquire(src_rows);
+    int64_t S64 = d_num[0], T = d_num[1];
+    const int S = (int)(S64 < 0 ? 0 : (S64 > (int64_t)S_max ? (int64_t)S_max : S64));
+    T = T < 0 ? 0 : (T < T_max ? T : T_max);
+    for (int s0 = blockIdx.x; s0 < S; s0 += gridDim.x) {
+        const int64_t begin = cu_seqlens[s0], end = cu_seqlens[s0 + 1];
+        if (end <= begin || end >= T) continue;                 // empty, or nothing follows
+        const int64_t t0 = (end - 1) / BM * BM;                 // tile of the survivor's last row
+        if (t0 < begin || t0 + BM <= end) continue;             // owned by an earlier survivor / ends with the tile
+        const int rows = (int)min((int64_t)BM, T - t0);
+        __syncthreads();                                        // src_row_of is free again
+        for (int r = threadIdx.x; r < rows; r += PACK_THREADS) {
+            const int64_t t = t0 + r;
+            int sv = s0;
+            while (sv + 1 < S && cu_seqlens[sv + 1] <= t) ++sv;
+            src_row_of[r] = src_tok_off[survivor_idx[sv]] + (t - cu_seqlens[sv]);
+        }
+        __syncthreads();
+        uint4* dst = scratch + (int64_t)s0 * BM * vec_per_row;
+        const int total = rows * vec_per_row;
+        for (int v0 = 0; v0 < total; v0 += 8 * PACK_THREADS) {
+            uint4 buf[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int vv = v0 + u * PACK_THREADS + threadIdx.x;
+                if (vv < total) {
+                    const int r = vv / vec_per_row;
+                    buf[u] = __ldg(src_rows + src_row_of[r] * vec_per_row + (vv - r * vec_per_row));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int vv = v0 + u * PACK_THREADS + threadIdx.x;
+                if (vv < total) dst[vv] = buf[u];
+            }
+        }
     }
 }
 
@@ -299,12 +412,17 @@ __global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, co
 
 // How many vocabulary splits per token tile.  With one split every resident block streams a different token
 // tile (128 x d x 2 bytes each) against the same W chunks; when those tiles together outgrow about half of L2
-// the tiles are re-fetched from HBM once per chunk, so the vocabulary is split until they fit (80 MB of the 126 MB L2).
+// the tiles are re-fetched from HBM once per chunk, so the vocabulary is split until they fit (40 MB of the 126 MB L2).
 int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
     const int total_chunks = (V + BN - 1) / BN;
     const int64_t m_tiles = (T_max + BM - 1) / BM;
     int splits = 1;
-    const double l2_budget = 80.0 * 1024 * 1024;   // measured: 74 MB of token tiles still stay L2-resident, 148 MB thrash
+    // Measured: 74 MB of token tiles stay L2-resident when they are one contiguous block (the packed rows) but not
+    // when they are scattered over a larger buffer (tiles read in place by the gathered variant: the SM clock under
+    // the power cap fell from 1.27 to 1.10 GHz with the extra HBM traffic); 37-47 MB stay resident either way, and
+    // the packed kernel runs the same cycles with the extra split.  One budget for both variants keeps their results
+    // bit-identical.
+    const double l2_budget = 40.0 * 1024 * 1024;
     const double tile_bytes = (double)BM * d * 2;
     while (splits < 8 && (ctx->sm_count / splits) * tile_bytes > l2_budget) splits *= 2;
     // few token tiles: split so that every SM has work
@@ -335,25 +453,47 @@ extern "C" int32_t arrol_token_logprob_splits(arrol_ctx* ctx, int64_t T_max, int
     return (total_chunks + chunks_per_split - 1) / chunks_per_split;
 }
 
+// Gather description of the gathered variant: the token rows come from `hidden` = the source buffer of
+// `source_rows` rows through (cu_seqlens, survivor_idx, src_tok_off); NULL = `hidden` is the packed [T_max, d] block.
+struct GatherArgs {
+    const int64_t* cu_seqlens;
+    const int32_t* survivor_idx;
+    const int64_t* src_tok_off;
+    const int64_t* d_num;
+    int64_t source_rows;
+    int32_t S_max;
+};
+
+// bytes of the boundary-tile scratch, placed after the split records in the gathered variant's workspace
+static size_t boundary_scratch_bytes(int32_t S_max, int32_t d) { return (size_t)S_max * BM * (size_t)d * 2; }
+
 static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
                              int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                              float* logp, float* lse, float* conf, void* workspace, size_t workspace_bytes,
-                             void* stream) {
+                             void* stream, const GatherArgs* ga = nullptr) {
     if (!ctx || T_max < 0 || d <= 0 || V <= 0 || !(inv_temperature > 0.f)) return ARROL_ERR_INVALID_ARG;
     if (T_max == 0) return ARROL_OK;
     if (!hidden || !W_vocab || !targets || !logp) return ARROL_ERR_INVALID_ARG;
     if (d % 8 != 0) return ARROL_ERR_UNSUPPORTED;
     if (!arrol_aligned(hidden, 16) || !arrol_aligned(W_vocab, 16)) return ARROL_ERR_INVALID_ARG;
     if (T_max > (int64_t)INT32_MAX - BM) return ARROL_ERR_UNSUPPORTED;   // TMA coordinates are 32-bit
-    const size_t need = arrol_token_logprob_workspace(ctx, T_max, d, V);
+    const size_t split_bytes = arrol_token_logprob_workspace(ctx, T_max, d, V);
+    const size_t need = split_bytes + (ga ? boundary_scratch_bytes(ga->S_max, d) : 0);
     if (!workspace || workspace_bytes < need || !arrol_aligned(workspace, 256)) return ARROL_ERR_WORKSPACE;
 
     ArrolDeviceGuard guard(ctx->device);
     if (!guard.ok) return ARROL_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
 
-    CUtensorMap map_h, map_w;
-    if (make_map(ctx, &map_h, hidden, (uint64_t)T_max, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    CUtensorMap map_h, map_s, map_w;
+    void* scratch = static_cast<uint8_t*>(workspace) + split_bytes;      // split_bytes is a multiple of 16 (256-aligned + records)
+    if (make_map(ctx, &map_h, hidden, (uint64_t)(ga ? ga->source_rows : T_max), (uint64_t)d, BM) != ARROL_OK)
+        return ARROL_ERR_CUDA;
+    if (ga) {
+        if (make_map(ctx, &map_s, scratch, (uint64_t)ga->S_max * BM, (uint64_t)d, BM) != ARROL_OK) return ARROL_ERR_CUDA;
+    } else {
+        map_s = map_h;
+    }
     if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
 
     LogprobParams p;
@@ -375,16 +515,35 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     p.d_status = ctx->d_status;
     p.spin_limit = ctx->test_spin_limit ? ctx->test_spin_limit : SPIN_LIMIT;
     p.mute_producer = ctx->test_mute_producer;
+    p.cu_seqlens = ga ? ga->cu_seqlens : nullptr;
+    p.survivor_idx = ga ? ga->survivor_idx : nullptr;
+    p.src_tok_off = ga ? ga->src_tok_off : nullptr;
+    p.d_num = ga ? ga->d_num : nullptr;
+    p.S_max = ga ? ga->S_max : 0;
+    p.timing = ctx->logprob_timing;
+    p.timing_items = ctx->logprob_timing_items;
 
-    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)SMEM_BYTES));
-    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)SMEM_BYTES));
     const int64_t m_tiles = (T_max + BM - 1) / BM;
     int64_t grid = m_tiles * p.splits;
     if (grid > ctx->sm_count) grid = ctx->sm_count;
-    if (conf) token_logprob_kernel<true><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
-    else token_logprob_kernel<false><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_w, p);
+    if (ga) {
+        int blocks = ga->S_max < ctx->sm_count * 4 ? ga->S_max : ctx->sm_count * 4;
+        ARROL_CUDA_OK(arrol_launch_pdl(pack_boundary_tiles_kernel, dim3((unsigned)blocks), dim3(PACK_THREADS), 0, s,
+                                       static_cast<const uint4*>(hidden), ga->cu_seqlens, ga->survivor_idx,
+                                       ga->src_tok_off, ga->d_num, ga->S_max, T_max, d / 8, static_cast<uint4*>(scratch)));
+        ctx->launches += 1;
+        token_logprob_kernel<false, true><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_s, map_w, p);
+    } else if (conf) {
+        token_logprob_kernel<true, false><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_s, map_w, p);
+    } else {
+        token_logprob_kernel<false, false><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_s, map_w, p);
+    }
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     if (p.splits > 1) {
@@ -413,4 +572,26 @@ extern "C" int arrol_token_logprob_conf(arrol_ctx* ctx, const void* hidden, cons
     if (T_max > 0 && !token_conf) return ARROL_ERR_INVALID_ARG;
     return run_token_logprob(ctx, hidden, W_vocab, targets, T_max, d_T, d, V, inv_temperature, logp, lse, token_conf,
                              workspace, workspace_bytes, stream);
+}
+
+extern "C" size_t arrol_token_logprob_gathered_workspace(arrol_ctx* ctx, int32_t S_max, int64_t T_max, int32_t d,
+                                                         int32_t V) {
+    if (!ctx || S_max <= 0 || T_max <= 0 || d <= 0 || V <= 0) return 0;
+    return arrol_token_logprob_workspace(ctx, T_max, d, V) + boundary_scratch_bytes(S_max, d);
+}
+
+extern "C" int arrol_token_logprob_gathered(arrol_ctx* ctx, const void* src_rows, int64_t source_rows,
+                                            const void* W_vocab, const int32_t* targets, const int64_t* cu_seqlens,
+                                            const int32_t* survivor_idx, const int64_t* src_tok_off,
+                                            const int64_t* d_num, int32_t S_max, int64_t T_max, int32_t d, int32_t V,
+                                            float inv_temperature, float* logp, float* lse, void* workspace,
+                                            size_t workspace_bytes, void* stream) {
+    if (!ctx || S_max < 0 || source_rows < 0 || T_max < 0) return ARROL_ERR_INVALID_ARG;
+    if (T_max == 0 || S_max == 0) return ARROL_OK;
+    if (!cu_seqlens || !survivor_idx || !src_tok_off || !d_num || source_rows == 0) return ARROL_ERR_INVALID_ARG;
+    if (source_rows > (int64_t)INT32_MAX - BM || (int64_t)S_max * BM > (int64_t)INT32_MAX - BM)
+        return ARROL_ERR_UNSUPPORTED;                                            // TMA coordinates are 32-bit
+    GatherArgs ga = {cu_seqlens, survivor_idx, src_tok_off, d_num, source_rows, S_max};
+    return run_token_logprob(ctx, src_rows, W_vocab, targets, T_max, d_num + 1, d, V, inv_temperature, logp, lse,
+                             nullptr, workspace, workspace_bytes, stream, &ga);
 }

@@ -77,7 +77,8 @@ class PruneRebatch:
         self.dst_rows = torch.empty((cap, w.d), dtype=torch.bfloat16, device=dev) if with_rows else None
         self.logp = torch.empty(cap, dtype=f32, device=dev)
         self.lse = torch.empty(cap, dtype=f32, device=dev)
-        ws = B.arrol_token_logprob_workspace(self.ctx, cap, w.d, w.V)
+        ws = max(B.arrol_token_logprob_workspace(self.ctx, cap, w.d, w.V),
+                 B.arrol_token_logprob_gathered_workspace(self.ctx, N, cap, w.d, w.V))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
 
     # ---- the four calls -------------------------------------------------------------------------------
@@ -100,6 +101,12 @@ class PruneRebatch:
         h = self.dst_rows if hidden is None else hidden
         B.arrol_token_logprob(self.ctx, h, self.W_vocab, self.dst_tokens, self.cap, self.w.d, self.w.V, self.logp,
                               self.workspace, lse=self.lse, d_T=self.d_num[1:])
+
+    def token_logprob_gathered(self):
+        """Log-probs with the survivors' rows read in place from the source buffer (no packed copy needed)."""
+        B.arrol_token_logprob_gathered(self.ctx, self.src_rows, self.W_vocab, self.dst_tokens, self.cu_seqlens,
+                                       self.survivor_idx, self.src_tok_off, self.d_num, self.w.N, self.cap, self.w.d,
+                                       self.w.V, self.logp, self.workspace, lse=self.lse)
 
     def prune_step(self, with_rows: Optional[bool] = None):
         self.score_partial()
