@@ -11,6 +11,16 @@
 //   warps 2..5  epilogue: thread r owns token row r of the tile; tcgen05.ld of its accumulator row, running
 //               maximum and sum of 2^(z log2e - max), and the target column's logit, all in registers
 // The two accumulators let the epilogue of chunk c overlap the MMAs of chunk c + 1.
+//
+// Waves in step.  The resident blocks all stream the same W_vocab chunks; as long as they do so at about the same
+// time a chunk comes from HBM once and from L2 147 times.  Nothing in a persistent kernel keeps them together,
+// though: measured on 6.5 M tokens (1,373 work items per block), the blocks' start times spread from 0.02 of an item
+// after two waves to 2 items after 50 and 40 items after 800; once a block lags by more than L2 holds it re-streams
+// its chunks from HBM, falls further behind, and the extra HBM traffic costs power: the SM clock under the 1 kW cap
+// fell from 1.40 GHz in the first waves to 0.72 GHz.  So the blocks are held in step: before issuing the loads of
+// wave k (its k-th work item) every producer arrives on a counter in global memory and waits until all blocks have
+// arrived for that wave.  The kernel is launched cooperatively whenever there is more than one wave, so that all
+// blocks are resident and the wait cannot deadlock; like every other wait it is bounded.
 // Every wait is bounded; when one runs out the block records ARROL_DEV_WAIT_EXPIRED, drains and returns.
 //
 // Gathered variant (arrol_token_logprob_gathered; Section 4.3 (ii): the survivors are re-batched "to compute
@@ -69,9 +79,16 @@ struct LogprobParams {
     const int64_t* src_tok_off;
     const int64_t* d_num;  // {S, T}
     int S_max;
+    unsigned int* wave_counter;   // producers that have arrived, over all waves of this launch (zeroed before it)
     unsigned long long* timing;   // test hook: per work item {globaltimer start, end, clock64 start, end}, or NULL
     int64_t timing_items;
 };
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
@@ -148,7 +165,25 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 const int64_t s64 = p.d_num[0];
                 S = (int)(s64 < 0 ? 0 : (s64 > (int64_t)p.S_max ? (int64_t)p.S_max : s64));
             }
-            for (int64_t item = blockIdx.x; item < items && ok && !p.mute_producer; item += gridDim.x) {
+            const int64_t waves = (items + gridDim.x - 1) / gridDim.x;
+            unsigned int wave = 0;
+            for (int64_t item = blockIdx.x; ok && !p.mute_producer; item += gridDim.x, ++wave) {
+                if (wave > 0 && wave < waves) {
+                    // hold the blocks in step: arrive for this wave, then wait for everybody (a block without a work
+                    // item in the last, partial wave arrives as well and leaves)
+                    __threadfence();
+                    atomicAdd(p.wave_counter, 1u);
+                    if (item < items) {
+                        const unsigned int target = wave * gridDim.x;
+                        uint32_t it = 0;
+                        while (ld_acquire_u32(p.wave_counter) < target) {
+                            __nanosleep(64);
+                            if (++it >= p.spin_limit || ((it & 1023u) == 1023u && *abort_flag)) { ok = false; break; }
+                        }
+                        if (!ok) { *abort_flag = 1u; break; }
+                    }
+                }
+                if (item >= items) break;
                 const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
                 const int c0 = split * p.chunks_per_split;
                 const int c1 = min(c0 + p.chunks_per_split, total_chunks);
@@ -520,6 +555,7 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     p.src_tok_off = ga ? ga->src_tok_off : nullptr;
     p.d_num = ga ? ga->d_num : nullptr;
     p.S_max = ga ? ga->S_max : 0;
+    p.wave_counter = ctx->d_tile_counters + ARROL_TILE_COUNTERS - 1;   // last word of the page: not a scoring counter
     p.timing = ctx->logprob_timing;
     p.timing_items = ctx->logprob_timing_items;
 
@@ -532,17 +568,30 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     const int64_t m_tiles = (T_max + BM - 1) / BM;
     int64_t grid = m_tiles * p.splits;
     if (grid > ctx->sm_count) grid = ctx->sm_count;
+    // more than one wave: the blocks wait for one another, so they must all be resident (cooperative launch)
+    const bool several_waves = m_tiles * p.splits > grid;
+    if (several_waves) ARROL_CUDA_OK(cudaMemsetAsync(p.wave_counter, 0, sizeof(unsigned int), s));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = several_waves ? 1 : 0;
     if (ga) {
         int blocks = ga->S_max < ctx->sm_count * 4 ? ga->S_max : ctx->sm_count * 4;
         ARROL_CUDA_OK(arrol_launch_pdl(pack_boundary_tiles_kernel, dim3((unsigned)blocks), dim3(PACK_THREADS), 0, s,
                                        static_cast<const uint4*>(hidden), ga->cu_seqlens, ga->survivor_idx,
                                        ga->src_tok_off, ga->d_num, ga->S_max, T_max, d / 8, static_cast<uint4*>(scratch)));
         ctx->launches += 1;
-        token_logprob_kernel<false, true><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_s, map_w, p);
+        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, true>, map_h, map_s, map_w, p));
     } else if (conf) {
-        token_logprob_kernel<true, false><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_s, map_w, p);
+        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<true, false>, map_h, map_s, map_w, p));
     } else {
-        token_logprob_kernel<false, false><<<(unsigned)grid, NUM_THREADS, SMEM_BYTES, s>>>(map_h, map_s, map_w, p);
+        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, false>, map_h, map_s, map_w, p));
     }
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());

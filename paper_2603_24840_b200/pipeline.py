@@ -6,7 +6,8 @@ synchronisation in between; the survivor token count stays on the device.  All a
 """
 from __future__ import annotations
 
-from typing import Dict, Optional
+import dataclasses
+from typing import Dict, List, Optional
 
 import numpy as np
 import torch
@@ -80,6 +81,53 @@ class PruneRebatch:
         ws = max(B.arrol_token_logprob_workspace(self.ctx, cap, w.d, w.V),
                  B.arrol_token_logprob_gathered_workspace(self.ctx, N, cap, w.d, w.V))
         self.workspace = torch.empty(ws, dtype=torch.uint8, device=dev)
+
+    @classmethod
+    def chunk_views(cls, parent: "PruneRebatch", n_chunks: int) -> List["PruneRebatch"]:
+        """Splits a resident workload into `n_chunks` groups of consecutive prompts that are processed one after the
+        other through ONE set of work buffers (packed rows, per-token arrays, workspace sized for the largest chunk).
+        Every view reads its own prompts' rows in the parent's source buffers (explicit offsets), so all of the
+        parent's prompts are covered and nothing is copied."""
+        w = parent.w
+        if w.P % n_chunks != 0:
+            raise ValueError("n_chunks must divide P")
+        Pc = w.P // n_chunks
+        Nc = Pc * w.G
+        wc = dataclasses.replace(w, P=Pc)
+        ell = parent.host["lengths"]
+        caps = [token_capacity(wc, ell[c * Nc:(c + 1) * Nc]) for c in range(n_chunks)]
+        cap = max(caps)
+        dev = parent.dev
+        i32, i64, f32 = torch.int32, torch.int64, torch.float32
+        ws = max(B.arrol_token_logprob_workspace(parent.ctx, cap, w.d, w.V),
+                 B.arrol_token_logprob_gathered_workspace(parent.ctx, Nc, cap, w.d, w.V))
+        bufs = dict(
+            score=torch.empty(Nc, dtype=f32, device=dev), prob=torch.empty(Nc, dtype=f32, device=dev),
+            q=torch.empty(Nc, dtype=f32, device=dev), bin=torch.empty(Nc, dtype=i32, device=dev),
+            keep=torch.empty(Nc, dtype=torch.uint8, device=dev), survivor_idx=torch.empty(Nc, dtype=i32, device=dev),
+            cu_seqlens=torch.empty(Nc + 1, dtype=i64, device=dev), adv=torch.empty(Nc, dtype=f32, device=dev),
+            dst_tokens=torch.empty(cap, dtype=i32, device=dev), tok_adv=torch.empty(cap, dtype=f32, device=dev),
+            tok_seq=torch.empty(cap, dtype=i32, device=dev),
+            dst_rows=torch.empty((cap, w.d), dtype=torch.bfloat16, device=dev),
+            logp=torch.empty(cap, dtype=f32, device=dev), lse=torch.empty(cap, dtype=f32, device=dev),
+            workspace=torch.empty(ws, dtype=torch.uint8, device=dev))
+        views = []
+        for c in range(n_chunks):
+            v = cls.__new__(cls)
+            sl = slice(c * Nc, (c + 1) * Nc)
+            v.w, v.dev, v.ctx, v.with_rows = wc, dev, parent.ctx, True
+            v.T_src, v.cap = parent.T_src, caps[c]
+            v.host = dict(parent.host, lengths=ell[sl], rewards=parent.host["rewards"][sl],
+                          src_tok_off=parent.host["src_tok_off"][c * Nc:(c + 1) * Nc + 1])
+            for name in ("lengths", "rewards", "src_tok_off", "row_index"):
+                setattr(v, name, getattr(parent, name)[sl])
+            for name in ("src_tokens", "head", "q_lut", "hidden_score", "src_rows", "W_vocab"):
+                setattr(v, name, getattr(parent, name))
+            for name, t in bufs.items():
+                setattr(v, name, t)
+            v.d_num = torch.zeros(2, dtype=i64, device=dev)      # every view keeps its own {S, T}
+            views.append(v)
+        return views
 
     # ---- the four calls -------------------------------------------------------------------------------
     def score_partial(self):

@@ -8,21 +8,33 @@ import torch
 
 import oracle
 from paper_2603_24840_b200 import binding as B
-from paper_2603_24840_b200 import dist_util, synth
+from paper_2603_24840_b200 import synth
 from paper_2603_24840_b200.pipeline import PruneRebatch, host_inputs
 
 pytestmark = pytest.mark.gpu
 
 
-def _fullsize(name, n_logp_rows, prompt_chunks=1):
+def _fullsize(name, n_logp_rows):
     w = synth.WORKLOADS[name]
-    if prompt_chunks > 1:                       # the benchmark runs this workload as chunks of P / prompt_chunks prompts
-        w = dist_util.shard_workload(w, 0, 1, prompt_chunks=prompt_chunks)
     inp = host_inputs(w)                       # big tensors are generated on the device
     pr = PruneRebatch(w, inputs=inp)
     pr.step()
     torch.cuda.synchronize()
     assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+    T = _check_state(pr, w, inp, n_logp_rows)
+    # the same step with the survivors' rows read in place (no packed copy): identical log-probs
+    ref = pr.logp[:T].clone()
+    pr.logp.fill_(7.0)
+    pr.prune_step(with_rows=False)
+    pr.token_logprob_gathered()
+    torch.cuda.synchronize()
+    assert pr.counts()[1] == T and torch.equal(pr.logp[:T], ref)
+    assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+    pr.ctx.close()
+
+
+def _check_state(pr, w, inp, n_logp_rows):
+    """Every output of a finished step of `pr` (a whole workload or one chunk view of it) against the oracle."""
     oa = lambda t: None if t is None else synth.as_oracle_array(t)
     head = inp["head"]
     off = inp["src_tok_off"]
@@ -86,7 +98,7 @@ def _fullsize(name, n_logp_rows, prompt_chunks=1):
     assert np.abs(logp[rows] - lp_ref).max() <= 2e-3
     assert np.abs(lse[rows] - lse_ref).max() <= 2e-3
     assert np.all(np.isfinite(logp)) and np.all(logp <= 1e-6) and np.all(logp > -60.0)
-    pr.ctx.close()
+    return T
 
 
 def test_llama_3_2_1b_shaped():
@@ -101,8 +113,28 @@ def test_qwen3_4b_shaped():
     _fullsize("qwen3-4b", 16)
 
 
-def test_qwen3_8b_dapo_shaped_one_prompt_chunk():
-    _fullsize("qwen3-8b-dapo", 16, prompt_chunks=4)
+def test_qwen3_8b_dapo_shaped_all_prompt_chunks_and_in_place():
+    """The largest workload as the benchmark runs it: all 256 prompts' source rows resident, four chunks of 64
+    different prompts through one set of packed buffers, every chunk checked; then all prompts in one pass with the
+    rows read in place, which must reproduce the chunks' log-probs bit for bit."""
+    w = synth.WORKLOADS["qwen3-8b-dapo"]
+    parent = PruneRebatch(w, inputs=host_inputs(w), with_rows=False)
+    views = PruneRebatch.chunk_views(parent, 4)
+    pieces, T_total = [], 0
+    for c, v in enumerate(views):
+        v.step()
+        torch.cuda.synchronize()
+        assert B.arrol_poll_status(parent.ctx, raise_on_error=False) == 0
+        T = _check_state(v, v.w, v.host, 12 if c in (0, 3) else 4)
+        pieces.append(v.logp[:T].clone())
+        T_total += T
+    parent.prune_step(with_rows=False)
+    parent.token_logprob_gathered()
+    torch.cuda.synchronize()
+    assert B.arrol_poll_status(parent.ctx, raise_on_error=False) == 0
+    assert parent.counts() == (w.S, T_total)
+    assert torch.equal(parent.logp[:T_total], torch.cat(pieces))
+    parent.ctx.close()
 
 
 def test_llama_3_2_1b_shaped_update_leg():
