@@ -17,6 +17,7 @@ struct arrol_ctx {
     float* d_scratch;          // MLP-head partial sums: [ARROL_SCRATCH_FLOATS]
     void* d_pack;              // MLP head on the tensor cores: the scored rows packed as bf16 [N][d], ARROL_PACK_BYTES
     uint32_t* d_tile_counters; // MLP head on the tensor cores: finished blocks per row tile, zero between calls
+    unsigned long long* d_chain;   // fused prune step: finished blocks, index-check flag, per-block totals; zero between calls
     bool score_tc_smem_set;    // the scoring kernel's dynamic shared-memory limit has been raised on this device
     bool gather_bulk_smem_set; // likewise for the bulk-copy gather kernel
     uint32_t test_spin_limit;  // arrol_test_hook: tries per pipeline wait of the log-prob kernel, 0 = the normal limit
@@ -37,7 +38,8 @@ constexpr int ARROL_MLP_TH = 64;             // hidden units per MLP thread-bloc
 constexpr int ARROL_MAX_H = 4096;
 constexpr size_t ARROL_SCRATCH_FLOATS = (size_t)ARROL_MAX_MLP_N * (ARROL_MAX_H / ARROL_MLP_TH);
 constexpr size_t ARROL_PACK_BYTES = (size_t)64 << 20;
-constexpr int ARROL_TILE_COUNTERS = 1024;
+constexpr int ARROL_TILE_COUNTERS = 1024;   // [0, 512) row tiles of the MLP head, [1023] log-prob waves
+constexpr int ARROL_CHAIN_BLOCKS = 510;      // blocks of the fused prune step's chained scan (2 + 2 * 510 words = 8 KB)
 
 #define ARROL_CUDA_OK(expr)                      \
     do {                                         \
@@ -100,6 +102,23 @@ cudaError_t arrol_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, si
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif
+
+// Argument checks of the three prune-step calls (score.cu, select.cu, compact.cu) and arrol_compact with the scan
+// kernel left out (the fused prune step has produced its outputs already).
+int arrol_internal_check_score(const void* hidden, int64_t row_stride_elems, int32_t N, const arrol_head* head,
+                               const arrol_calib* calib, const float* score, const float* prob, const float* q);
+int arrol_internal_check_select(const float* q, int32_t P, int32_t G, int32_t K, double rho, int32_t mode,
+                                const uint8_t* keep);
+int arrol_internal_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths, const int64_t* src_tok_off,
+                           int32_t N, int32_t G, const int32_t* src_tokens, const void* src_rows, int32_t row_bytes,
+                           const float* rewards, float eps, int32_t ddof, int64_t dst_capacity_tokens,
+                           int32_t* dst_tokens, void* dst_rows, int64_t* cu_seqlens, int32_t* survivor_idx, float* adv,
+                           float* tok_adv, int32_t* tok_seq, int64_t* d_num, void* stream, bool scan_done);
+int arrol_internal_check_compact(const uint8_t* keep, const int32_t* lengths, const int64_t* src_tok_off, int32_t N,
+                                 int32_t G, const int32_t* src_tokens, const void* src_rows, int32_t row_bytes,
+                                 const float* rewards, float eps, int32_t ddof, int64_t dst_capacity_tokens,
+                                 const int32_t* dst_tokens, const void* dst_rows, const int64_t* cu_seqlens,
+                                 const int32_t* survivor_idx, const float* adv, const int64_t* d_num);
 
 // score.cu: MLP tile pass with optional pre-activation output; partial is [ceil(h / ARROL_MLP_TH)][N].
 int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const int64_t* row_index, int N,

@@ -11,13 +11,9 @@
 //   cu_seqlens), then the block streams the tile's payload with 16-byte loads/stores, eight in flight per thread.
 //   T is read from device memory, so there is no host synchronisation between the kernels.
 #include "arrol_internal.h"
+#include "prune_kernels.cuh"
 
 namespace {
-
-constexpr int SCAN_THREADS = 1024;
-constexpr int SCAN_ITEMS = 4;      // consecutive rollouts per thread and pass: N <= 4096 is one pass
-constexpr int SCAN_INV = 65;
-constexpr int SCAN_GROUPS = SCAN_THREADS * SCAN_ITEMS / 4 + 2;   // groups of size >= 4 that one pass can touch
 
 __global__ void __launch_bounds__(SCAN_THREADS)
 scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ lengths, int N, int G,
@@ -25,174 +21,12 @@ scan_adv_kernel(const uint8_t* __restrict__ keep, const int32_t* __restrict__ le
                 int32_t* __restrict__ survivor_idx, int64_t* __restrict__ cu_seqlens, float* __restrict__ adv,
                 int64_t* __restrict__ d_num, uint32_t* __restrict__ d_status,
                 const int64_t* __restrict__ src_tok_off, int64_t source_rows) {
-    __shared__ int32_t warp_cnt[32];
-    __shared__ int64_t warp_tok[32];
-    // per-group statistics of the groups a pass touches (G >= 4: at most SCAN_GROUPS of them)
-    __shared__ double g_mean[SCAN_GROUPS], g_den[SCAN_GROUPS];     // mean, 1 / (std + eps)
-    // the pass's keep flags and rewards, staged once so that the statistics and the advantages read shared memory
-    __shared__ float s_rew[SCAN_THREADS * SCAN_ITEMS];
-    __shared__ uint8_t s_keep[SCAN_THREADS * SCAN_ITEMS];
-    __shared__ double s_inv[SCAN_INV];             // 1 / count for the small counts
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const bool shared_stats = G >= 4;
     pdl_launch_dependents();
     pdl_wait();
     keep = pdl_acquire(keep); lengths = pdl_acquire(lengths); rewards = pdl_acquire(rewards);
     src_tok_off = pdl_acquire(src_tok_off);
-    if (threadIdx.x == 0) cu_seqlens[0] = 0;
-    bool bad_index = false;          // a kept rollout whose source rows leave the caller's buffer (checked on request)
-    int32_t carry_c = 0;             // survivors / tokens of the passes so far (the same in every thread)
-    int64_t carry_t = 0;
-
-    // statistics over the kept rollouts of a group (Section 3, on survivors): sums in index order, fp64
-    constexpr int PASS = SCAN_THREADS * SCAN_ITEMS;
-    // Statistics of group g over its kept rollouts: mean and 1 / (std + eps), in fp64.  A double-precision division
-    // or square root costs this one-block kernel about half a microsecond each, so the reciprocals of the small
-    // counts come from a table and sqrt / reciprocal are Newton steps from single-precision seeds (relative error
-    // below 1e-15 after two steps); values outside the single-precision range take the plain operations.
-    // inv_den = 0 (advantage exactly 0) when fewer than ddof + 1 rollouts are kept or all kept rewards are equal.
-    auto group_stats = [&](int g, int base, double& mean, double& inv_den) {
-        const int g0 = g * G;
-        const int g1 = min(g0 + G, N);
-        // members inside the staged pass come from shared memory, a group that straddles its edge reads the rest
-        // from global memory; the loads do not depend on the flags, so they overlap; adding 0.0 for a pruned
-        // rollout changes nothing
-        auto flag = [&](int r) { return (unsigned)(r - base) < (unsigned)PASS ? s_keep[r - base] != 0 : keep[r] != 0; };
-        auto rew = [&](int r) { return (unsigned)(r - base) < (unsigned)PASS ? s_rew[r - base] : rewards[r]; };
-        int n = 0;
-        double sum = 0.0;
-        float first = 0.f;
-        bool all_equal = true;
-#pragma unroll 4
-        for (int r = g0; r < g1; ++r) {
-            const bool k = flag(r);
-            const float v = rew(r);
-            if (k && n == 0) first = v;
-            all_equal = all_equal && (!k || v == first);
-            sum += k ? (double)v : 0.0;
-            n += k ? 1 : 0;
-        }
-        auto recip_count = [&](int c) { return c < SCAN_INV ? s_inv[c] : 1.0 / (double)c; };
-        mean = n > 0 ? sum * recip_count(n) : 0.0;
-        double ss = 0.0;
-#pragma unroll 4
-        for (int r = g0; r < g1; ++r) {
-            const bool k = flag(r);
-            const double dv = (double)rew(r) - mean;
-            ss += k ? dv * dv : 0.0;
-        }
-        inv_den = 0.0;
-        if (n - ddof > 0 && !all_equal) {
-            const double var = ss * recip_count(n - ddof);
-            double sd;
-            const float varf = (float)var;
-            if (varf > 1e-30f && varf < 1e30f) {
-                double y = (double)rsqrtf(varf);
-                y = y * (1.5 - 0.5 * var * y * y);
-                y = y * (1.5 - 0.5 * var * y * y);
-                sd = var * y;
-            } else {
-                sd = sqrt(var);
-            }
-            const double den = sd + eps;
-            const float denf = (float)den;
-            if (denf > 1e-30f && denf < 1e30f) {
-                double x = (double)(1.0f / denf);
-                x = x * (2.0 - den * x);
-                x = x * (2.0 - den * x);
-                inv_den = x;
-            } else {
-                inv_den = 1.0 / den;
-            }
-        }
-    };
-
-    if (threadIdx.x >= 1 && threadIdx.x < SCAN_INV) s_inv[threadIdx.x] = 1.0 / (double)threadIdx.x;   // before the first barrier below
-
-    for (int base = 0; base < N; base += PASS) {
-        const int i0 = base + threadIdx.x * SCAN_ITEMS;
-        bool kept[SCAN_ITEMS];
-        int64_t len[SCAN_ITEMS];
-        int32_t c = 0;
-        int64_t t = 0;
-        // one round of coalesced loads: flags and rewards of the pass into shared memory, lengths into registers
-        for (int e = threadIdx.x; e < PASS; e += SCAN_THREADS) {
-            const int i = base + e;
-            s_keep[e] = i < N ? keep[i] : (uint8_t)0;
-            s_rew[e] = i < N ? rewards[i] : 0.f;
-        }
-#pragma unroll
-        for (int u = 0; u < SCAN_ITEMS; ++u) len[u] = (i0 + u < N) ? (int64_t)max(lengths[i0 + u], 0) : 0;
-        __syncthreads();
-#pragma unroll
-        for (int u = 0; u < SCAN_ITEMS; ++u) {
-            kept[u] = s_keep[threadIdx.x * SCAN_ITEMS + u] != 0;
-            if (!kept[u]) len[u] = 0;
-            else if (source_rows > 0) {
-                const int64_t o = src_tok_off[i0 + u];
-                bad_index = bad_index || o < 0 || o + len[u] > source_rows;
-            }
-        }
-        const int g_lo = base / G;
-        if (shared_stats) {          // one thread per group of this pass; visible after the scan's first barrier
-            const int g_hi = (min(N, base + PASS) - 1) / G;
-            for (int gi = threadIdx.x; gi <= g_hi - g_lo; gi += SCAN_THREADS)
-                group_stats(g_lo + gi, base, g_mean[gi], g_den[gi]);
-        }
-#pragma unroll
-        for (int u = 0; u < SCAN_ITEMS; ++u) { c += kept[u] ? 1 : 0; t += len[u]; }
-        const int32_t own_c = c;
-        const int64_t own_t = t;
-        // inclusive scan of the per-thread totals inside the warp
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int32_t oc = __shfl_up_sync(0xffffffffu, c, o);
-            const int64_t ot = __shfl_up_sync(0xffffffffu, t, o);
-            if (lane >= o) { c += oc; t += ot; }
-        }
-        if (lane == 31) { warp_cnt[wid] = c; warp_tok[wid] = t; }
-        __syncthreads();
-        // every warp scans the 32 warp totals itself (no second barrier, no single-warp phase)
-        int32_t wc = warp_cnt[lane];
-        int64_t wt = warp_tok[lane];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int32_t oc = __shfl_up_sync(0xffffffffu, wc, o);
-            const int64_t ot = __shfl_up_sync(0xffffffffu, wt, o);
-            if (lane >= o) { wc += oc; wt += ot; }
-        }
-        const int32_t pass_cnt = __shfl_sync(0xffffffffu, wc, 31);          // totals of the pass
-        const int64_t pass_tok = __shfl_sync(0xffffffffu, wt, 31);
-        const int32_t before_c = __shfl_sync(0xffffffffu, wc, wid ? wid - 1 : 0);
-        const int64_t before_t = __shfl_sync(0xffffffffu, wt, wid ? wid - 1 : 0);
-        int32_t pos = carry_c + (wid ? before_c : 0) + (c - own_c);   // survivors before this thread's items
-        int64_t tok = carry_t + (wid ? before_t : 0) + (t - own_t);
-#pragma unroll
-        for (int u = 0; u < SCAN_ITEMS; ++u) {
-            if (!kept[u]) continue;
-            const int i = i0 + u;
-            tok += len[u];
-            survivor_idx[pos] = i;
-            cu_seqlens[pos + 1] = tok;
-            double mean, den;
-            if (shared_stats) { mean = g_mean[i / G - g_lo]; den = g_den[i / G - g_lo]; }
-            else group_stats(i / G, base, mean, den);
-            const double a = ((double)s_rew[i - base] - mean) * den;      // den holds 1 / (std + eps), or 0
-            adv[pos] = (float)a;
-            ++pos;
-        }
-        carry_c += pass_cnt;
-        carry_t += pass_tok;
-        __syncthreads();                 // the staging arrays and warp totals are rewritten by the next pass
-    }
-    const int any_bad = __syncthreads_or(bad_index ? 1 : 0);
-    if (threadIdx.x == 0) {
-        d_num[0] = carry_c;
-        d_num[1] = carry_t;
-        if (carry_t > capacity) atomicOr(d_status, ARROL_DEV_CAPACITY);
-        if (any_bad) atomicOr(d_status, ARROL_DEV_BAD_INDEX);
-        d_status[1] = any_bad ? 1u : 0u;       // gate word: the gather kernels of this call copy nothing when it is set
-    }
+    scan_adv_block(keep, lengths, N, G, rewards, eps, ddof, capacity, survivor_idx, cu_seqlens, adv, d_num, d_status,
+                   src_tok_off, source_rows);
 }
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
@@ -336,13 +170,13 @@ gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restric
 
 }  // namespace
 
-extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths,
-                             const int64_t* src_tok_off, int32_t N, int32_t G, const int32_t* src_tokens,
-                             const void* src_rows, int32_t row_bytes, const float* rewards, float eps,
-                             int32_t ddof, int64_t dst_capacity_tokens, int32_t* dst_tokens, void* dst_rows,
-                             int64_t* cu_seqlens, int32_t* survivor_idx, float* adv, float* tok_adv,
-                             int32_t* tok_seq, int64_t* d_num, void* stream) {
-    if (!ctx || N < 0 || G < 1 || dst_capacity_tokens < 0 || ddof < 0 || !(eps >= 0.f)) return ARROL_ERR_INVALID_ARG;
+// Argument checks of arrol_compact, shared with arrol_prune_step's fused path.
+int arrol_internal_check_compact(const uint8_t* keep, const int32_t* lengths, const int64_t* src_tok_off, int32_t N,
+                                 int32_t G, const int32_t* src_tokens, const void* src_rows, int32_t row_bytes,
+                                 const float* rewards, float eps, int32_t ddof, int64_t dst_capacity_tokens,
+                                 const int32_t* dst_tokens, const void* dst_rows, const int64_t* cu_seqlens,
+                                 const int32_t* survivor_idx, const float* adv, const int64_t* d_num) {
+    if (N < 0 || G < 1 || dst_capacity_tokens < 0 || ddof < 0 || !(eps >= 0.f)) return ARROL_ERR_INVALID_ARG;
     if (!cu_seqlens || !d_num) return ARROL_ERR_INVALID_ARG;
     if (N > 0 && (!keep || !lengths || !src_tok_off || !rewards || !survivor_idx || !adv))
         return ARROL_ERR_INVALID_ARG;
@@ -354,13 +188,32 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
         if (row_bytes % 16 != 0) return ARROL_ERR_UNSUPPORTED;
         if (!arrol_aligned(src_rows, 16) || !arrol_aligned(dst_rows, 16)) return ARROL_ERR_INVALID_ARG;
     }
+    return ARROL_OK;
+}
+
+// arrol_compact with the scan kernel optional: the fused prune step has already produced the scan outputs.
+int arrol_internal_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths,
+                             const int64_t* src_tok_off, int32_t N, int32_t G, const int32_t* src_tokens,
+                             const void* src_rows, int32_t row_bytes, const float* rewards, float eps,
+                             int32_t ddof, int64_t dst_capacity_tokens, int32_t* dst_tokens, void* dst_rows,
+                             int64_t* cu_seqlens, int32_t* survivor_idx, float* adv, float* tok_adv,
+                             int32_t* tok_seq, int64_t* d_num, void* stream, bool scan_done) {
+    if (!ctx) return ARROL_ERR_INVALID_ARG;
+    {
+        const int rc = arrol_internal_check_compact(keep, lengths, src_tok_off, N, G, src_tokens, src_rows, row_bytes,
+                                                    rewards, eps, ddof, dst_capacity_tokens, dst_tokens, dst_rows,
+                                                    cu_seqlens, survivor_idx, adv, d_num);
+        if (rc != ARROL_OK) return rc;
+    }
     ArrolDeviceGuard guard(ctx->device);
     if (!guard.ok) return ARROL_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
-    ARROL_CUDA_OK(arrol_launch_pdl(scan_adv_kernel, dim3(1), dim3(SCAN_THREADS), 0, s, keep, lengths, N, G, rewards,
-                                   (double)eps, ddof, dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
-                                   ctx->d_status, src_tok_off, ctx->source_rows));
-    ctx->launches += 1;
+    if (!scan_done) {
+        ARROL_CUDA_OK(arrol_launch_pdl(scan_adv_kernel, dim3(1), dim3(SCAN_THREADS), 0, s, keep, lengths, N, G, rewards,
+                                       (double)eps, ddof, dst_capacity_tokens, survivor_idx, cu_seqlens, adv, d_num,
+                                       ctx->d_status, src_tok_off, ctx->source_rows));
+        ctx->launches += 1;
+    }
     const bool any_token_output = dst_tokens || dst_rows || tok_adv || tok_seq;
     if (N == 0 || dst_capacity_tokens == 0 || !any_token_output) return ARROL_OK;
 
@@ -402,4 +255,15 @@ extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t*
                                    static_cast<uint4*>(dst_rows), tok_adv, tok_seq, ctx->d_status + 1));
     ctx->launches += 1;
     return ARROL_OK;
+}
+
+extern "C" int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths,
+                             const int64_t* src_tok_off, int32_t N, int32_t G, const int32_t* src_tokens,
+                             const void* src_rows, int32_t row_bytes, const float* rewards, float eps,
+                             int32_t ddof, int64_t dst_capacity_tokens, int32_t* dst_tokens, void* dst_rows,
+                             int64_t* cu_seqlens, int32_t* survivor_idx, float* adv, float* tok_adv,
+                             int32_t* tok_seq, int64_t* d_num, void* stream) {
+    return arrol_internal_compact(ctx, keep, lengths, src_tok_off, N, G, src_tokens, src_rows, row_bytes, rewards, eps,
+                                  ddof, dst_capacity_tokens, dst_tokens, dst_rows, cu_seqlens, survivor_idx, adv, tok_adv,
+                                  tok_seq, d_num, stream, false);
 }

@@ -44,6 +44,7 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->d_scratch = nullptr;
     ctx->d_pack = nullptr;
     ctx->d_tile_counters = nullptr;
+    ctx->d_chain = nullptr;
     ctx->score_tc_smem_set = false;
     ctx->gather_bulk_smem_set = false;
     ctx->test_spin_limit = 0;
@@ -64,6 +65,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
               cudaMalloc(&ctx->d_pack, ARROL_PACK_BYTES) == cudaSuccess &&
               cudaMalloc(&ctx->d_tile_counters, ARROL_TILE_COUNTERS * sizeof(uint32_t)) == cudaSuccess &&
               cudaMemset(ctx->d_tile_counters, 0, ARROL_TILE_COUNTERS * sizeof(uint32_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->d_chain, (2 + 2 * ARROL_CHAIN_BLOCKS) * sizeof(unsigned long long)) == cudaSuccess &&
+              cudaMemset(ctx->d_chain, 0, (2 + 2 * ARROL_CHAIN_BLOCKS) * sizeof(unsigned long long)) == cudaSuccess &&
               cudaMallocHost(&ctx->h_keep, ARROL_MAX_HOST_N) == cudaSuccess &&
               cudaMallocHost(&ctx->h_stage, ARROL_STAGE_BYTES) == cudaSuccess &&
               cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
@@ -93,6 +96,7 @@ extern "C" int arrol_destroy(arrol_ctx* ctx) {
     if (ctx->d_scratch) (void)cudaFree(ctx->d_scratch);
     if (ctx->d_pack) (void)cudaFree(ctx->d_pack);
     if (ctx->d_tile_counters) (void)cudaFree(ctx->d_tile_counters);
+    if (ctx->d_chain) (void)cudaFree(ctx->d_chain);
     if (ctx->h_keep) (void)cudaFreeHost(ctx->h_keep);
     if (ctx->h_stage) (void)cudaFreeHost(ctx->h_stage);
     for (int i = 0; i < ARROL_COPY_EVENTS; ++i)

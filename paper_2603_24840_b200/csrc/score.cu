@@ -11,50 +11,10 @@
 #include <cuda_bf16.h>
 
 #include "arrol_internal.h"
+#include "prune_kernels.cuh"
 #include "score_common.cuh"
 
 namespace {
-
-__device__ __forceinline__ float to_f32(float v) { return v; }
-__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __bfloat162float(v); }
-
-// 16-byte vector of T -> floats
-template <typename T> struct Vec16;
-template <> struct Vec16<float> {
-    static constexpr int N = 4;
-    using Raw = float4;
-    __device__ static __forceinline__ Raw load_raw(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
-    __device__ static __forceinline__ float dot(const Raw& a, const Raw& b, float acc) {
-        acc = fmaf(a.x, b.x, acc); acc = fmaf(a.y, b.y, acc); acc = fmaf(a.z, b.z, acc); return fmaf(a.w, b.w, acc);
-    }
-    __device__ static __forceinline__ void load(const float* p, float (&out)[4]) {
-        float4 v = __ldg(reinterpret_cast<const float4*>(p));
-        out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
-    }
-};
-template <> struct Vec16<__nv_bfloat16> {
-    static constexpr int N = 8;
-    using Raw = uint4;
-    __device__ static __forceinline__ Raw load_raw(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
-    __device__ static __forceinline__ float dot(const Raw& a, const Raw& b, float acc) {
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {   // a bf16 is the upper half of a binary32
-            acc = fmaf(__uint_as_float(aw[i] << 16), __uint_as_float(bw[i] << 16), acc);
-            acc = fmaf(__uint_as_float(aw[i] & 0xffff0000u), __uint_as_float(bw[i] & 0xffff0000u), acc);
-        }
-        return acc;
-    }
-    __device__ static __forceinline__ void load(const __nv_bfloat16* p, float (&out)[8]) {
-        uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {   // a bf16 is the upper half of a binary32
-            out[2 * i] = __uint_as_float(w[i] << 16);
-            out[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-    }
-};
 
 template <typename T>
 __global__ void __launch_bounds__(128)
@@ -77,25 +37,7 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
         if (lane == 0) atomicOr(d_status, ARROL_DEV_BAD_INDEX);
         nvec = 0;
     }
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    // eight independent 16-byte loads of x (and of w) in flight per lane: a 4 KB row is one round trip
-    for (int c0 = lane; c0 < nvec; c0 += 256) {
-        typename Vec16<T>::Raw xr[8], wr[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int c = c0 + 32 * u;
-            if (c < nvec) {
-                xr[u] = Vec16<T>::load_raw(x + (int64_t)c * VN);
-                wr[u] = Vec16<T>::load_raw(w + (int64_t)c * VN);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (c0 + 32 * u < nvec) acc[u & 3] = Vec16<T>::dot(xr[u], wr[u], acc[u & 3]);
-    }
-    float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    float s = linear_row_dot<T>(x, w, nvec, lane);
     if (lane == 0) {
         if (bias) s += to_f32(bias[0]);
         probability_map(s, warp, B, q_lut, score, prob, bin, q);
@@ -364,12 +306,33 @@ int arrol_internal_mlp_tiles(arrol_ctx* ctx, const void* hidden, int64_t row_str
     return ARROL_OK;
 }
 
+// Argument checks of arrol_score_partial (N > 0), shared with arrol_prune_step's fused path.
+int arrol_internal_check_score(const void* hidden, int64_t row_stride_elems, int32_t N, const arrol_head* head,
+                               const arrol_calib* calib, const float* score, const float* prob, const float* q) {
+    if (!hidden || !score || !prob || !q || !head->W1) return ARROL_ERR_INVALID_ARG;
+    if (head->dtype != ARROL_F32 && head->dtype != ARROL_BF16) return ARROL_ERR_INVALID_ARG;
+    if (head->d <= 0 || head->h < 0) return ARROL_ERR_INVALID_ARG;
+    if (head->h > 0 && !head->w2) return ARROL_ERR_INVALID_ARG;
+    const int esz = head->dtype == ARROL_F32 ? 4 : 2;
+    if (head->d % 8 != 0 || head->h % 4 != 0 || head->h > ARROL_MAX_H) return ARROL_ERR_UNSUPPORTED;
+    if (head->h > 0 && N > ARROL_MAX_MLP_N) return ARROL_ERR_UNSUPPORTED;
+    if (row_stride_elems < head->d) return ARROL_ERR_INVALID_ARG;
+    if (!arrol_aligned(hidden, 16) || !arrol_aligned(head->W1, 16) || (row_stride_elems * esz) % 16 != 0)
+        return ARROL_ERR_INVALID_ARG;
+    if (calib && calib->q_lut && calib->B <= 0) return ARROL_ERR_INVALID_ARG;
+    return ARROL_OK;
+}
+
 extern "C" int arrol_score_partial(arrol_ctx* ctx, const void* hidden, int64_t row_stride_elems,
                                    const int64_t* row_index, int32_t N, const arrol_head* head,
                                    const arrol_calib* calib, float* score, float* prob, int32_t* bin, float* q,
                                    void* stream) {
     if (!ctx || !head || N < 0) return ARROL_ERR_INVALID_ARG;
     if (N == 0) return ARROL_OK;
+    {
+        const int rc = arrol_internal_check_score(hidden, row_stride_elems, N, head, calib, score, prob, q);
+        if (rc != ARROL_OK) return rc;
+    }
     if (!hidden || !score || !prob || !q || !head->W1) return ARROL_ERR_INVALID_ARG;
     if (head->dtype != ARROL_F32 && head->dtype != ARROL_BF16) return ARROL_ERR_INVALID_ARG;
     if (head->d <= 0 || head->h < 0) return ARROL_ERR_INVALID_ARG;

@@ -7,22 +7,9 @@
 // higher index wins, then the winner leaves the group and Sigma -= q_winner.  Sigma starts as the index-order
 // sum, built with broadcasts so that every lane of the segment adds the same values in the same order.
 #include "arrol_internal.h"
+#include "prune_kernels.cuh"
 
 namespace {
-
-__device__ __forceinline__ double shfl_double(double v, int src_lane, int width) {
-    int lo = __double2loint(v), hi = __double2hiint(v);
-    lo = __shfl_sync(0xffffffffu, lo, src_lane, width);
-    hi = __shfl_sync(0xffffffffu, hi, src_lane, width);
-    return __hiloint2double(hi, lo);
-}
-
-__device__ __forceinline__ double shfl_xor_double(double v, int mask, int width) {
-    int lo = __double2loint(v), hi = __double2hiint(v);
-    lo = __shfl_xor_sync(0xffffffffu, lo, mask, width);
-    hi = __shfl_xor_sync(0xffffffffu, hi, mask, width);
-    return __hiloint2double(hi, lo);
-}
 
 __global__ void __launch_bounds__(128)
 select_kernel(const float* __restrict__ q, int P, int G, int K, double rho, int seg, uint8_t* __restrict__ keep) {
@@ -35,42 +22,30 @@ select_kernel(const float* __restrict__ q, int P, int G, int K, double rho, int 
     const int j = lane & (seg - 1);                       // index inside the group
     const int group = warp * groups_per_warp + lane / seg;
     const bool member = (group < P) && (j < G);
-
     const double qj = member ? (double)q[(int64_t)group * G + j] : 0.0;
-    bool alive = member;
-
-    double sigma = 0.0;
-    for (int i = 0; i < G; ++i) sigma = __dadd_rn(sigma, shfl_double(qj, i, seg));
-
-    for (int n = G; n > K; --n) {
-        const double tau = __dsub_rn(sigma, __dmul_rn(rho, (double)(n - 1)));
-        double key = alive ? fabs(__dsub_rn(qj, tau)) : __longlong_as_double(0x7ff0000000000000LL);
-        int idx = alive ? j : -1;
-        // segmented arg-min; ties -> the higher index
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            if (o < seg) {
-                const double okey = shfl_xor_double(key, o, seg);
-                const int oidx = __shfl_xor_sync(0xffffffffu, idx, o, seg);
-                if (okey < key || (okey == key && oidx > idx)) { key = okey; idx = oidx; }
-            }
-        }
-        const double q_removed = shfl_double(qj, idx < 0 ? 0 : idx, seg);
-        if (idx == j) alive = false;
-        sigma = __dsub_rn(sigma, q_removed);
-    }
+    const bool alive = select_lanes(qj, member, j, G, K, rho, seg);
     if (member) keep[(int64_t)group * G + j] = alive ? 1 : 0;
 }
 
 }  // namespace
+// Argument checks of arrol_select, shared with arrol_prune_step's fused path.
+int arrol_internal_check_select(const float* q, int32_t P, int32_t G, int32_t K, double rho, int32_t mode,
+                                const uint8_t* keep) {
+    if (P < 0 || G < 1 || K < 1 || K > G) return ARROL_ERR_INVALID_ARG;
+    if (mode != 0 || G > 32) return ARROL_ERR_UNSUPPORTED;
+    if (!(rho >= 0.0 && rho <= 1.0)) return ARROL_ERR_INVALID_ARG;
+    if (P > 0 && (!q || !keep)) return ARROL_ERR_INVALID_ARG;
+    return ARROL_OK;
+}
 
 extern "C" int arrol_select(arrol_ctx* ctx, const float* q, int32_t P, int32_t G, int32_t K, double rho,
                             int32_t mode, uint8_t* keep, void* stream) {
-    if (!ctx || P < 0 || G < 1 || K < 1 || K > G) return ARROL_ERR_INVALID_ARG;
-    if (mode != 0 || G > 32) return ARROL_ERR_UNSUPPORTED;
-    if (!(rho >= 0.0 && rho <= 1.0)) return ARROL_ERR_INVALID_ARG;
+    if (!ctx) return ARROL_ERR_INVALID_ARG;
+    {
+        const int rc = arrol_internal_check_select(q, P, G, K, rho, mode, keep);
+        if (rc != ARROL_OK) return rc;
+    }
     if (P == 0) return ARROL_OK;
-    if (!q || !keep) return ARROL_ERR_INVALID_ARG;
     int seg = 1;
     while (seg < G) seg <<= 1;
     const int groups_per_warp = 32 / seg;
