@@ -34,9 +34,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic of one token_logprob launch per survivor token, by (d, V, vocabulary splits), from a single-launch
 # profiler capture on the small Llama-shaped case: (bytes read + bytes written) / tokens of the launch.  At fixed
 # d, V and split count the traffic grows in proportion to the tokens of the launch.
-LOGPROB_DRAM_BYTES_PER_TOKEN = {}
+LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256, 2): 60016.0}
 # DRAM bytes per scored row of score_linear_kernel streamed over consecutive rows (same kind of capture)
-SCORE_LINEAR_DRAM_BYTES_PER_ROW = {}
+SCORE_LINEAR_DRAM_BYTES_PER_ROW = {(2048, 2): 4129.8}
 
 
 def logprob_traffic(w, T, splits, sm_count):
@@ -876,6 +876,40 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_profile_leg(args, w):
+    """One call of the path a few times on a small workload, for single-kernel profiler captures: the state is built
+    and a whole step run twice, then the named call three times.  Prints how the call was made."""
+    import torch
+    from paper_2603_24840_b200 import binding as B
+    from paper_2603_24840_b200.pipeline import PruneRebatch
+    pr = PruneRebatch(w, device=0, with_rows=True)
+    for _ in range(2):
+        pr.step()
+    torch.cuda.synchronize()
+    n_stream = min(pr.T_src, 1 << 20)
+    so = [torch.empty(n_stream, dtype=torch.float32, device=pr.dev) for _ in range(3)]
+    step_args = pr.prune_step_args(with_rows=False)
+    legs = {
+        "score_stream": lambda: B.arrol_score_partial(pr.ctx, pr.hidden_score, pr.head, n_stream, so[0], so[1], so[2],
+                                                      q_lut=pr.q_lut),
+        "score": pr.score_partial,
+        "select": pr.select,
+        "compact": pr.compact,
+        "compact_tokens": lambda: pr.compact(False),
+        "logprob": pr.token_logprob,
+        "logprob_gathered": pr.token_logprob_gathered,
+        "prune_step": lambda: B.arrol_prune_step(pr.ctx, step_args),
+    }
+    fn = legs[args.profile_leg]
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    S, T = pr.counts()
+    B.arrol_poll_status(pr.ctx)
+    print(json.dumps({"profile_leg": args.profile_leg, "workload": w.name, "calls": 3, "N": w.N, "survivors": S,
+                      "survivor_tokens": T, "source_rows": pr.T_src, "streamed_rows": n_stream, "d": w.d, "V": w.V}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -890,10 +924,14 @@ def main():
     ap.add_argument("--skip-aux", action="store_true", help="leave out the timings of the calls around the step")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiler captures)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
+    ap.add_argument("--profile-leg", default=None, help="run one call of the path three times (for profiler captures): "
+                    "score_stream, score, select, compact, compact_tokens, logprob, logprob_gathered, prune_step")
     args = ap.parse_args()
     from paper_2603_24840_b200 import synth
     w = synth.WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.profile_leg:
+        run_profile_leg(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         if args.warmup < 3:

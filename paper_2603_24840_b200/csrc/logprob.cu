@@ -447,17 +447,20 @@ __global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, co
 
 // How many vocabulary splits per token tile.  With one split every resident block streams a different token
 // tile (128 x d x 2 bytes each) against the same W chunks; when those tiles together outgrow about half of L2
-// the tiles are re-fetched from HBM once per chunk, so the vocabulary is split until they fit (40 MB of the 126 MB L2).
+// the tiles are re-fetched from HBM once per chunk, so the vocabulary is split until they fit.
 int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
     const int total_chunks = (V + BN - 1) / BN;
     const int64_t m_tiles = (T_max + BM - 1) / BM;
-    int splits = 1;
-    // Measured: 74 MB of token tiles stay L2-resident when they are one contiguous block (the packed rows) but not
-    // when they are scattered over a larger buffer (tiles read in place by the gathered variant: the SM clock under
-    // the power cap fell from 1.27 to 1.10 GHz with the extra HBM traffic); 37-47 MB stay resident either way, and
-    // the packed kernel runs the same cycles with the extra split.  One budget for both variants keeps their results
-    // bit-identical.
-    const double l2_budget = 40.0 * 1024 * 1024;
+    // Measured with the blocks in step (TFLOP/s, packed rows / rows read in place by the gathered variant):
+    //   d = 2048: 1 split (148 resident tiles, 74 MB) 1,380 / 1,200;  2 splits (74 tiles, 37 MB) 1,377 / 1,378
+    //   d = 2560: 1 split (95 MB) 1,041 / 1,070;  2 splits (47 MB) 1,392 / 1,391;  4 splits (24 MB) 1,362 / 1,362
+    //   d = 4096: 1 split (148 MB) 990 / 987;  2 splits (74 MB) 1,391 / 1,377;  4 splits (37 MB) 1,363 / 1,363
+    // Token tiles beyond what L2 keeps are re-fetched from HBM once per chunk; every split beyond that streams
+    // W_vocab from HBM once more per wave.  So: two splits whenever there is a full wave of tiles (tiles read in place
+    // are scattered over the source buffer and 148 of them do not stay resident even at 74 MB), more only while the
+    // resident tiles exceed 80 MB.  One rule for both variants keeps their results bit-identical.
+    int splits = m_tiles >= ctx->sm_count ? 2 : 1;
+    const double l2_budget = 80.0 * 1024 * 1024;
     const double tile_bytes = (double)BM * d * 2;
     while (splits < 8 && (ctx->sm_count / splits) * tile_bytes > l2_budget) splits *= 2;
     // few token tiles: split so that every SM has work
