@@ -3,7 +3,9 @@ at a barrier and when the timings are reduced (max over ranks) and the processed
 from __future__ import annotations
 
 import dataclasses
+from typing import List, Sequence, Tuple
 
+import numpy as np
 import torch
 import torch.distributed as dist
 
@@ -28,3 +30,27 @@ def reduce_timings(step_ms: float, e2e_ms: float, tokens: float, device) -> tupl
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.all_reduce(n, op=dist.ReduceOp.SUM)
     return float(t[0]), float(t[1]), float(n[0])
+
+
+def balanced_partition(group_tokens: Sequence[int], world: int) -> List[Tuple[int, int]]:
+    """Contiguous ranges [begin, end) of prompt groups for `world` ranks, balanced by token count: `group_tokens[g]`
+    is the work of group g (the sum of its rollouts' lengths before pruning, its survivor tokens after).  Greedy on
+    the prefix sums: rank r ends at the group whose prefix sum is nearest to (r + 1) / world of the total, with at
+    least one group per rank while groups remain.  Groups stay whole and in order, so no exchange is needed."""
+    t = np.asarray(group_tokens, dtype=np.int64)
+    n = int(t.shape[0])
+    if world < 1:
+        raise ValueError("world must be positive")
+    prefix = np.concatenate([[0], np.cumsum(t)])
+    total = int(prefix[-1])
+    bounds = [0]
+    for r in range(world - 1):
+        target = total * (r + 1) / world
+        lo = min(bounds[-1] + 1, n)                            # at least one group, if any is left
+        hi = max(lo, n - (world - 1 - r))                      # leave one group for every later rank where possible
+        cut = int(np.searchsorted(prefix, target, side="left"))
+        if cut > 0 and abs(prefix[cut - 1] - target) <= abs(prefix[min(cut, n)] - target):
+            cut -= 1
+        bounds.append(int(min(max(cut, lo), max(hi, lo))) if lo <= n else n)
+    bounds.append(n)
+    return [(bounds[r], bounds[r + 1]) for r in range(world)]

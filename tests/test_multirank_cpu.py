@@ -64,3 +64,32 @@ def test_shard_workload_properties():
     w5 = synth.WORKLOADS["qwen3-8b-dapo"]
     assert dist_util.shard_workload(w5, 0, 1, prompt_chunks=4).P == w5.P // 4
     assert dist_util.reduce_timings(1.0, 2.0, 3.0, "cpu") == (1.0, 2.0, 3.0)   # no process group: identity
+
+
+def test_token_balanced_partition_of_the_prompt_groups():
+    """Contiguous, complete, ordered ranges; imbalance (max / mean tokens per rank) small on the five workloads, both
+    before pruning (sum of lengths per group) and after (the K longest rollouts of a group as a stand-in for its
+    survivors)."""
+    import numpy as np
+    from paper_2603_24840_b200 import dist_util, synth
+    for name in synth.WORKLOAD_ORDER:
+        w = synth.WORKLOADS[name]
+        ell = synth.lengths(w).astype(np.int64).reshape(w.P, w.G)
+        for tokens in (ell.sum(1), np.sort(ell, axis=1)[:, -w.K:].sum(1)):
+            for world in (1, 2, 3, 4, 8):
+                if world > w.P:
+                    continue
+                parts = dist_util.balanced_partition(tokens, world)
+                assert parts[0][0] == 0 and parts[-1][1] == w.P
+                assert all(parts[r][1] == parts[r + 1][0] for r in range(world - 1))
+                assert all(b < e for b, e in parts)
+                per_rank = np.array([tokens[b:e].sum() for b, e in parts])
+                # never worse than one (largest) group above the even share
+                assert per_rank.max() <= tokens.sum() / world + tokens.max()
+                if w.P >= 16 * world:
+                    assert per_rank.max() / per_rank.mean() <= 1.10
+    # degenerate inputs
+    assert dist_util.balanced_partition([5, 5], 1) == [(0, 2)]
+    assert dist_util.balanced_partition([], 2) == [(0, 0), (0, 0)]
+    assert dist_util.balanced_partition([7], 3) == [(0, 1), (1, 1), (1, 1)]
+    assert dist_util.balanced_partition([1, 1, 100, 1, 1], 2) in ([(0, 2), (2, 5)], [(0, 3), (3, 5)])
