@@ -458,11 +458,18 @@ int64_t arrol_launch_count(arrol_ctx* ctx);
  *                                    {globaltimer at start, globaltimer at end, SM clock at start, SM clock at end}
  *                                    of its epilogue, from which a benchmark derives the SM clock the kernel ran at
  *                                    (cycles / nanoseconds) without reading or setting any GPU clock control.
+ *   ARROL_HOOK_LOGPROB_SPLITS        value = vocabulary splits per token tile (1..64; 0 = chosen from the sizes, the
+ *                                    default); set it before sizing the workspace, which depends on it.
+ *   ARROL_HOOK_LOGPROB_PAIR          value != 0 (the default): the log-prob kernel runs as clusters of two thread blocks
+ *                                    that share one 256-row tile (tcgen05 cta_group::2); 0: one block per 128-row tile.
+ *                                    Set it before sizing the workspace, which depends on it.
  * Returns INVALID_ARG for an unknown key or a limit outside [0, 2^26]. */
 #define ARROL_HOOK_SPIN_LIMIT 1
 #define ARROL_HOOK_MUTE_LOGPROB_PRODUCER 2
 #define ARROL_HOOK_LOGPROB_TIMING_BUFFER 3
 #define ARROL_HOOK_LOGPROB_TIMING_ITEMS 4
+#define ARROL_HOOK_LOGPROB_PAIR 5
+#define ARROL_HOOK_LOGPROB_SPLITS 6
 int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value);
 
 #ifdef __cplusplus

@@ -297,7 +297,7 @@ def arrol_token_logprob_gathered(ctx: Context, src_rows, W_vocab, targets, cu_se
         _stream(stream)), "arrol_token_logprob_gathered")
 
 
-HOOK_SPIN_LIMIT, HOOK_MUTE_LOGPROB_PRODUCER, HOOK_LOGPROB_TIMING_BUFFER, HOOK_LOGPROB_TIMING_ITEMS = 1, 2, 3, 4
+HOOK_SPIN_LIMIT, HOOK_MUTE_LOGPROB_PRODUCER, HOOK_LOGPROB_TIMING_BUFFER, HOOK_LOGPROB_TIMING_ITEMS, HOOK_LOGPROB_PAIR, HOOK_LOGPROB_SPLITS = 1, 2, 3, 4, 5, 6
 
 
 def arrol_test_hook(ctx: Context, key: int, value: int):

@@ -49,6 +49,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->gather_bulk_smem_set = false;
     ctx->test_spin_limit = 0;
     ctx->test_mute_producer = 0;
+    ctx->logprob_pair = 1;
+    ctx->logprob_splits = 0;
     ctx->logprob_timing = nullptr;
     ctx->logprob_timing_items = 0;
     ctx->encode_tiled = nullptr;
@@ -123,6 +125,13 @@ extern "C" int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value) {
             return ARROL_OK;
         case ARROL_HOOK_MUTE_LOGPROB_PRODUCER:
             ctx->test_mute_producer = value != 0;
+            return ARROL_OK;
+        case ARROL_HOOK_LOGPROB_SPLITS:
+            if (value < 0 || value > 64) return ARROL_ERR_INVALID_ARG;
+            ctx->logprob_splits = (int)value;
+            return ARROL_OK;
+        case ARROL_HOOK_LOGPROB_PAIR:
+            ctx->logprob_pair = value != 0;
             return ARROL_OK;
         case ARROL_HOOK_LOGPROB_TIMING_BUFFER:
             ctx->logprob_timing = reinterpret_cast<unsigned long long*>((uintptr_t)value);

@@ -44,14 +44,21 @@ namespace {
 
 constexpr int BM = 128;          // token rows per tile  (MMA M)
 constexpr int BN = 256;          // vocabulary columns per chunk (MMA N)
-constexpr int STAGES = 4;
+constexpr int SOLO_STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
-constexpr int B_STAGE_BYTES = BN * BK * 2;   // 32 KB
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int SOLO_B_STAGE_BYTES = BN * BK * 2;   // 32 KB
+constexpr int SOLO_STAGE_BYTES = A_STAGE_BYTES + SOLO_B_STAGE_BYTES;
+// pair variant (two blocks of a cluster on one 256-row tile): every block stages its 128 rows of A and its half of
+// the B tile, so a stage is 32 KB and six of them fit
+constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_B_ROWS = BN / 2;
+constexpr int PAIR_B_STAGE_BYTES = PAIR_B_ROWS * BK * 2;   // 16 KB
+constexpr int PAIR_STAGE_BYTES = A_STAGE_BYTES + PAIR_B_STAGE_BYTES;
+static_assert(PAIR_STAGES * PAIR_STAGE_BYTES == SOLO_STAGES * SOLO_STAGE_BYTES, "both variants fill the same shared memory");
 constexpr int TMEM_COLS = 512;   // two fp32 accumulators of BN columns
 constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr size_t SMEM_BYTES = (size_t)SOLO_STAGES * SOLO_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 
 struct PartialLse {   // per (split, token): running maximum and sum in the base-2 domain, target logit,
     float m2, l, zy2, pad;   // pad: sum of the raw accumulators of the split (only when the confidence is asked for)
@@ -108,17 +115,25 @@ __device__ __forceinline__ int survivor_of_row(const int64_t* __restrict__ cu_se
 
 // GATHER: map_h covers the pre-prune source rows and map_s the scratch of pre-packed boundary tiles
 // ([S_max * 128, d], slot s at rows 128 s ...); otherwise map_h covers the packed rows and map_s is unused.
-template <bool CONF, bool GATHER>
+// PAIR: the kernel runs as clusters of two blocks; a pair works on 256 token rows (block r of the pair owns rows
+// 128 r ...), block 0 issues 256 x 256 x 16 MMAs (cta_group::2) that read both blocks' shared memory and write both
+// blocks' tensor memory, every block loads its own 128 rows of A and its own 128 of the chunk's 256 W_vocab rows and
+// runs the epilogue of its own rows.  Per block and K step 32 KB come in from L2 instead of 48 KB and the tensor
+// core reads 8 KB of operands per MMA from shared memory instead of 12 KB.
+template <bool CONF, bool GATHER, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_s,
                      const __grid_constant__ CUtensorMap map_w, const LogprobParams p) {
+    constexpr int STAGES = PAIR ? PAIR_STAGES : SOLO_STAGES;
+    constexpr int B_STAGE_BYTES = PAIR ? PAIR_B_STAGE_BYTES : SOLO_B_STAGE_BYTES;
+    constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
     extern __shared__ uint8_t smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle pattern
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* stage_a = smem;
     uint8_t* stage_b = smem + (size_t)STAGES * A_STAGE_BYTES;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
-    uint64_t* full = bars;                    // [STAGES]  TMA -> MMA
+    uint64_t* full = bars;                    // [STAGES]  TMA -> MMA (pair: block 0's receive both blocks' bytes)
     uint64_t* empty = bars + STAGES;          // [STAGES]  MMA -> TMA
     uint64_t* acc_full = bars + 2 * STAGES;   // [2]       MMA -> epilogue
     uint64_t* acc_empty = acc_full + 2;       // [2]       epilogue -> MMA
@@ -127,17 +142,22 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // pair: rank of this block in its cluster (block 0 leads), unit = cluster; otherwise unit = block
+    const uint32_t rank = PAIR ? cluster_cta_rank() : 0u;
+    const int64_t unit = PAIR ? (int64_t)(blockIdx.x >> 1) : (int64_t)blockIdx.x;
+    const int64_t units = PAIR ? (int64_t)(gridDim.x >> 1) : (int64_t)gridDim.x;
 
     int64_t T = p.T_max;
     if (p.d_T) { const int64_t t = *p.d_T; T = t < 0 ? 0 : (t < T ? t : T); }
     const int64_t m_tiles = (T + BM - 1) / BM;
-    const int64_t items = m_tiles * p.splits;
+    const int64_t items = (PAIR ? (m_tiles + 1) / 2 : m_tiles) * p.splits;   // (pairs of) token tiles x splits
     const int k_steps = (p.d + BK - 1) / BK;
     const int total_chunks = (p.V + BN - 1) / BN;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], EPI_THREADS / 32); }
+        // pair: the leading block's acc_empty collects the epilogue warps of both blocks
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], (PAIR ? 2 : 1) * (EPI_THREADS / 32)); }
         mbar_init(drain, 1);
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -146,13 +166,20 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
         if constexpr (GATHER) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_s) : "memory");
     }
     if (warp == 1) {
-        tcgen05_alloc(tmem_slot, TMEM_COLS);
-        tcgen05_relinquish();
+        if constexpr (PAIR) { tcgen05_alloc_pair(tmem_slot, TMEM_COLS); tcgen05_relinquish_pair(); }
+        else { tcgen05_alloc(tmem_slot, TMEM_COLS); tcgen05_relinquish(); }
     }
     tcgen05_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();     // the peer's barriers exist before anything arrives on them
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // pair: shared::cluster addresses, in the leading block, of the barriers both blocks signal
+    uint32_t lead_full0 = 0, lead_acc_empty0 = 0;
+    if constexpr (PAIR) {
+        lead_full0 = map_to_cta(smem_u32(&full[0]), 0u);
+        lead_acc_empty0 = map_to_cta(smem_u32(&acc_empty[0]), 0u);
+    }
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -165,16 +192,18 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 const int64_t s64 = p.d_num[0];
                 S = (int)(s64 < 0 ? 0 : (s64 > (int64_t)p.S_max ? (int64_t)p.S_max : s64));
             }
-            const int64_t waves = (items + gridDim.x - 1) / gridDim.x;
+            const int64_t waves = (items + units - 1) / units;
             unsigned int wave = 0;
-            for (int64_t item = blockIdx.x; ok && !p.mute_producer; item += gridDim.x, ++wave) {
+            for (int64_t item = unit; ok && !p.mute_producer; item += units, ++wave) {
                 if (wave > 0 && wave < waves) {
-                    // hold the blocks in step: arrive for this wave, then wait for everybody (a block without a work
-                    // item in the last, partial wave arrives as well and leaves)
-                    __threadfence();
-                    atomicAdd(p.wave_counter, 1u);
+                    // hold the blocks in step: arrive for this wave (one arrival per unit), then wait for everybody (a
+                    // unit without a work item in the last, partial wave arrives as well and leaves)
+                    if (rank == 0) {
+                        __threadfence();
+                        atomicAdd(p.wave_counter, 1u);
+                    }
                     if (item < items) {
-                        const unsigned int target = wave * gridDim.x;
+                        const unsigned int target = wave * (unsigned int)units;
                         uint32_t it = 0;
                         while (ld_acquire_u32(p.wave_counter) < target) {
                             __nanosleep(64);
@@ -184,7 +213,8 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                     }
                 }
                 if (item >= items) break;
-                const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
+                const int tile_unit = (int)(item / p.splits), split = (int)(item % p.splits);
+                const int m_tile = PAIR ? 2 * tile_unit + (int)rank : tile_unit;      // this block's 128 rows
                 const int c0 = split * p.chunks_per_split;
                 const int c1 = min(c0 + p.chunks_per_split, total_chunks);
                 // where the tile's 128 rows come from: the packed rows, a run of source rows, or a scratch slot
@@ -192,29 +222,43 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 int a_row = m_tile * BM;
                 if constexpr (GATHER) {
                     const int64_t t0 = (int64_t)m_tile * BM;
-                    const int s0 = survivor_of_row(p.cu_seqlens, S, t0);
-                    const int64_t s_end = p.cu_seqlens[s0 + 1];
-                    if (s_end < t0 + BM && s_end < T) {     // the tile runs on into the next survivor: pre-packed
-                        a_map = &map_s;
-                        a_row = s0 * BM;
-                    } else {
-                        a_row = (int)(p.src_tok_off[p.survivor_idx[s0]] + (t0 - p.cu_seqlens[s0]));
+                    a_row = 0;                              // a pair's second tile may lie past T: any rows will do
+                    if (t0 < T) {
+                        const int s0 = survivor_of_row(p.cu_seqlens, S, t0);
+                        const int64_t s_end = p.cu_seqlens[s0 + 1];
+                        if (s_end < t0 + BM && s_end < T) {     // the tile runs on into the next survivor: pre-packed
+                            a_map = &map_s;
+                            a_row = s0 * BM;
+                        } else {
+                            a_row = (int)(p.src_tok_off[p.survivor_idx[s0]] + (t0 - p.cu_seqlens[s0]));
+                        }
                     }
                 }
                 for (int c = c0; c < c1 && ok; ++c) {
                     for (int ks = 0; ks < k_steps; ++ks) {
                         if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
-                        mbar_expect_tx(&full[stage], STAGE_BYTES);
-                        tma_load_2d(stage_a + (size_t)stage * A_STAGE_BYTES, a_map, ks * BK, a_row, &full[stage]);
-                        tma_load_2d(stage_b + (size_t)stage * B_STAGE_BYTES, &map_w, ks * BK, c * BN, &full[stage]);
+                        if constexpr (PAIR) {
+                            // both blocks' bytes are counted on the leading block's barrier
+                            const uint32_t bar = lead_full0 + stage * (uint32_t)sizeof(uint64_t);
+                            if (rank == 0) mbar_expect_tx(&full[stage], 2 * STAGE_BYTES);
+                            tma_load_2d_pair(stage_a + (size_t)stage * A_STAGE_BYTES, a_map, ks * BK, a_row, bar);
+                            tma_load_2d_pair(stage_b + (size_t)stage * B_STAGE_BYTES, &map_w, ks * BK,
+                                             c * BN + (int)rank * PAIR_B_ROWS, bar);
+                        } else {
+                            mbar_expect_tx(&full[stage], STAGE_BYTES);
+                            tma_load_2d(stage_a + (size_t)stage * A_STAGE_BYTES, a_map, ks * BK, a_row, &full[stage]);
+                            tma_load_2d(stage_b + (size_t)stage * B_STAGE_BYTES, &map_w, ks * BK, c * BN, &full[stage]);
+                        }
                         ++issued;
                         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
-            if (!ok) {
+            if (!ok && rank == 0) {
                 // Gave up: let the copies already issued land before the block's shared memory goes away.
-                // The last min(issued, STAGES) stages may still be in flight; wait for each (bounded).
+                // The last min(issued, STAGES) stages may still be in flight; wait for each (bounded).  (In a pair the
+                // second block's copies are counted on the leading block's barriers; the cluster barrier at the end
+                // of the kernel keeps its shared memory alive until the leading block has got here.)
                 const uint32_t pending = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
                 uint32_t s = stage, ph = phase;
                 for (uint32_t i = 0; i < pending; ++i) {
@@ -226,12 +270,12 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BM, BN);
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc(PAIR ? 2 * BM : BM, BN);
             uint32_t stage = 0, phase = 0;
             uint32_t acc = 0, acc_phase = 0;
             bool ok = true;
-            for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            for (int64_t item = unit; item < items && ok; item += units) {
                 const int split = (int)(item % p.splits);
                 const int c0 = split * p.chunks_per_split;
                 const int c1 = min(c0 + p.chunks_per_split, total_chunks);
@@ -247,19 +291,29 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
 #pragma unroll
                         for (int k = 0; k < BK / UMMA_K; ++k) {
                             // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in address units
-                            tcgen05_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                             (ks | k) != 0 ? 1u : 0u);
+                            if constexpr (PAIR)
+                                tcgen05_mma_bf16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                                      (ks | k) != 0 ? 1u : 0u);
+                            else
+                                tcgen05_mma_bf16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                                 (ks | k) != 0 ? 1u : 0u);
                         }
-                        tcgen05_commit(&empty[stage]);   // stage reusable once these MMAs have read it
+                        // stage reusable (in both blocks of a pair) once these MMAs have read it
+                        if constexpr (PAIR) tcgen05_commit_pair(&empty[stage], (uint16_t)3);
+                        else tcgen05_commit(&empty[stage]);
                         if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                     }
-                    if (ok) tcgen05_commit(&acc_full[acc]);   // accumulator complete
+                    if (ok) {                                 // accumulator complete
+                        if constexpr (PAIR) tcgen05_commit_pair(&acc_full[acc], (uint16_t)3);
+                        else tcgen05_commit(&acc_full[acc]);
+                    }
                     if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
                 }
             }
             if (!ok) {
                 // Gave up: wait (bounded) until the MMAs already issued have finished with shared and tensor memory.
-                tcgen05_commit(drain);
+                if constexpr (PAIR) tcgen05_commit_pair(drain, (uint16_t)1);
+                else tcgen05_commit(drain);
                 for (uint32_t it = 0; it < p.spin_limit; ++it)
                     if (mbar_try_wait(drain, 0u)) break;
             }
@@ -271,14 +325,15 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        for (int64_t item = blockIdx.x; item < items && ok; item += gridDim.x) {
-            const int m_tile = (int)(item / p.splits), split = (int)(item % p.splits);
+        for (int64_t item = unit; item < items && ok; item += units) {
+            const int tile_unit = (int)(item / p.splits), split = (int)(item % p.splits);
+            const int m_tile = PAIR ? 2 * tile_unit + (int)rank : tile_unit;
             const int c0 = split * p.chunks_per_split;
             const int c1 = min(c0 + p.chunks_per_split, total_chunks);
             const int64_t t = (int64_t)m_tile * BM + row_in_tile;
             const int y = (t < T) ? p.targets[t] : -1;
             float m2 = -INFINITY, l = 0.f, zy2 = -INFINITY, sumz = 0.f;
-            const bool stamp = p.timing != nullptr && threadIdx.x == 64 && item < p.timing_items;
+            const bool stamp = p.timing != nullptr && threadIdx.x == 64 && rank == 0 && item < p.timing_items;
             if (stamp) { p.timing[4 * item] = global_timer_ns(); p.timing[4 * item + 2] = (unsigned long long)clock64(); }
             for (int c = c0; c < c1 && ok; ++c) {
                 ok = mbar_wait(&acc_full[acc], acc_phase, abort_flag, p.spin_limit);
@@ -324,7 +379,10 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
                 }
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&acc_empty[acc]);
+                if (lane == 0) {
+                    if constexpr (PAIR) mbar_arrive_cluster(lead_acc_empty0 + acc * (uint32_t)sizeof(uint64_t));
+                    else mbar_arrive(&acc_empty[acc]);
+                }
                 if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
             if (stamp) { p.timing[4 * item + 1] = global_timer_ns(); p.timing[4 * item + 3] = (unsigned long long)clock64(); }
@@ -352,10 +410,12 @@ token_logprob_kernel(const __grid_constant__ CUtensorMap map_h, const __grid_con
 
     tcgen05_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();     // neither block's shared or tensor memory goes away under the other
     if (threadIdx.x == 0 && *abort_flag) atomicOr(p.d_status, ARROL_DEV_WAIT_EXPIRED);
     if (warp == 1) {
         tcgen05_fence_after();
-        tcgen05_dealloc(tmem_base, TMEM_COLS);
+        if constexpr (PAIR) tcgen05_dealloc_pair(tmem_base, TMEM_COLS);
+        else tcgen05_dealloc(tmem_base, TMEM_COLS);
     }
 }
 
@@ -455,12 +515,18 @@ int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
     //   d = 2048: 1 split (148 resident tiles, 74 MB) 1,380 / 1,200;  2 splits (74 tiles, 37 MB) 1,377 / 1,378
     //   d = 2560: 1 split (95 MB) 1,041 / 1,070;  2 splits (47 MB) 1,392 / 1,391;  4 splits (24 MB) 1,362 / 1,362
     //   d = 4096: 1 split (148 MB) 990 / 987;  2 splits (74 MB) 1,391 / 1,377;  4 splits (37 MB) 1,363 / 1,363
+    // and as pairs of blocks (cta_group::2), same order:
+    //   d = 2048: 1 split 1,389 / 1,271;  2 splits 1,411-1,427 / 1,403-1,410
+    //   d = 2560: 2 splits 1,428 / 1,413;  4 splits 1,403 / 1,396
+    //   d = 4096: 2 splits (74 MB) 1,235 / 1,232;  4 splits (37 MB) 1,392 / 1,371;  8 splits 1,357 / 1,352
     // Token tiles beyond what L2 keeps are re-fetched from HBM once per chunk; every split beyond that streams
     // W_vocab from HBM once more per wave.  So: two splits whenever there is a full wave of tiles (tiles read in place
     // are scattered over the source buffer and 148 of them do not stay resident even at 74 MB), more only while the
-    // resident tiles exceed 80 MB.  One rule for both variants keeps their results bit-identical.
+    // resident tiles exceed 80 MB (one block per tile) or 50 MB (pairs).  The packed and the in-place variant follow
+    // the same rule, so their results are bit-identical.
+    if (ctx->logprob_splits > 0) return ctx->logprob_splits < total_chunks ? ctx->logprob_splits : total_chunks;
     int splits = m_tiles >= ctx->sm_count ? 2 : 1;
-    const double l2_budget = 80.0 * 1024 * 1024;
+    const double l2_budget = (ctx->logprob_pair ? 50.0 : 80.0) * 1024 * 1024;
     const double tile_bytes = (double)BM * d * 2;
     while (splits < 8 && (ctx->sm_count / splits) * tile_bytes > l2_budget) splits *= 2;
     // few token tiles: split so that every SM has work
@@ -532,7 +598,9 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     } else {
         map_s = map_h;
     }
-    if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, BN) != ARROL_OK) return ARROL_ERR_CUDA;
+    // pair variant (clusters of two blocks): every block loads half of a chunk's W_vocab rows
+    const bool pair = ctx->logprob_pair != 0 && ctx->sm_count >= 2;
+    if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, pair ? PAIR_B_ROWS : BN) != ARROL_OK) return ARROL_ERR_CUDA;
 
     LogprobParams p;
     p.targets = targets;
@@ -562,39 +630,63 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     p.timing = ctx->logprob_timing;
     p.timing_items = ctx->logprob_timing_items;
 
-    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)SMEM_BYTES));
-    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)SMEM_BYTES));
-    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, false, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true, false, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, true, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, false, true>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<false, true, true>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true, false, true>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     const int64_t m_tiles = (T_max + BM - 1) / BM;
-    int64_t grid = m_tiles * p.splits;
-    if (grid > ctx->sm_count) grid = ctx->sm_count;
+    // work items and the units that take them: blocks, or pairs of blocks on 256 rows
+    const int64_t items_max = (pair ? (m_tiles + 1) / 2 : m_tiles) * p.splits;
+    int64_t units = pair ? ctx->sm_count / 2 : ctx->sm_count;
+    if (units > items_max) units = items_max;
+    const int64_t grid = pair ? 2 * units : units;
     // more than one wave: the blocks wait for one another, so they must all be resident (cooperative launch)
-    const bool several_waves = m_tiles * p.splits > grid;
+    const bool several_waves = items_max > units;
     if (several_waves) ARROL_CUDA_OK(cudaMemsetAsync(p.wave_counter, 0, sizeof(unsigned int), s));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (several_waves) {
+        attr[n_attr].id = cudaLaunchAttributeCooperative;
+        attr[n_attr].val.cooperative = 1;
+        ++n_attr;
+    }
+    if (pair) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 2;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = several_waves ? 1 : 0;
+    cfg.numAttrs = n_attr;
     if (ga) {
         int blocks = ga->S_max < ctx->sm_count * 4 ? ga->S_max : ctx->sm_count * 4;
         ARROL_CUDA_OK(arrol_launch_pdl(pack_boundary_tiles_kernel, dim3((unsigned)blocks), dim3(PACK_THREADS), 0, s,
                                        static_cast<const uint4*>(hidden), ga->cu_seqlens, ga->survivor_idx,
                                        ga->src_tok_off, ga->d_num, ga->S_max, T_max, d / 8, static_cast<uint4*>(scratch)));
         ctx->launches += 1;
-        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, true>, map_h, map_s, map_w, p));
+        if (pair) ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, true, true>, map_h, map_s, map_w, p));
+        else ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, true, false>, map_h, map_s, map_w, p));
     } else if (conf) {
-        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<true, false>, map_h, map_s, map_w, p));
+        if (pair) ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<true, false, true>, map_h, map_s, map_w, p));
+        else ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<true, false, false>, map_h, map_s, map_w, p));
+    } else if (pair) {
+        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, false, true>, map_h, map_s, map_w, p));
     } else {
-        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, false>, map_h, map_s, map_w, p));
+        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, false, false>, map_h, map_s, map_w, p));
     }
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());

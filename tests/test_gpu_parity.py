@@ -447,3 +447,35 @@ def test_whole_path_tiny():
 
 def test_whole_path_mini():
     _pipeline_parity("mini", None)
+
+
+@pytest.mark.parametrize("T,d,V,splits", [(300, 64, 300, 0), (1000, 192, 3000, 0), (128 * 148 * 2 + 77, 64, 520, 0),
+                                          (128 * 148 + 5, 64, 1100, 3), (700, 128, 2000, 2)])
+def test_pairs_of_blocks_and_single_blocks_give_the_same_logprobs(T, d, V, splits):
+    """The log-prob kernel as clusters of two blocks on 256-row tiles (the default) against one block per 128-row tile:
+    the same products in the same order, so the same bits; both within 2e-3 of the oracle.  Covers a single partial
+    wave, several waves (the blocks wait for one another per wave), an odd number of token tiles, forced splits."""
+    ctx = B.Context(0)
+    if splits:
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_SPLITS, splits)
+    g = np.random.default_rng(T + V)
+    H = torch.from_numpy(g.normal(size=(T, d)).astype(np.float32)).to(torch.bfloat16)
+    W = torch.from_numpy(g.normal(0, 0.05, size=(V, d)).astype(np.float32)).to(torch.bfloat16)
+    y = g.integers(0, V, size=T).astype(np.int32)
+    out = []
+    for pair in (1, 0):
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, pair)
+        ws = torch.empty(B.arrol_token_logprob_workspace(ctx, T, d, V), dtype=torch.uint8, device="cuda")
+        lp = torch.full((T,), 7.0, device="cuda")
+        lse = torch.full((T,), 7.0, device="cuda")
+        B.arrol_token_logprob(ctx, H.cuda(), W.cuda(), dev(y), T, d, V, lp, ws, lse=lse)
+        torch.cuda.synchronize()
+        out.append((lp, lse))
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
+    assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1])
+    rows = np.unique(np.concatenate([[0, T - 1, min(T - 1, 127), min(T - 1, 128), min(T - 1, 255), min(T - 1, 256)],
+                                     g.integers(0, T, size=40)])).astype(np.int64)
+    lp_ref, lse_ref = oracle.token_logprob(synth.as_oracle_array(H), synth.as_oracle_array(W), y, rows=rows)
+    assert np.abs(out[0][0].cpu().numpy()[rows] - lp_ref).max() <= LOGP_TOL
+    assert np.abs(out[0][1].cpu().numpy()[rows] - lse_ref).max() <= LOGP_TOL
+    ctx.close()
