@@ -180,6 +180,23 @@ def scored_rows_of(w):
     return synth.hidden_states(w, w.N, stream=21), "rows drawn on the host (no CUDA device to regenerate the GPU arm's)"
 
 
+_ORACLE_INPUTS = {}
+
+
+def oracle_inputs(w):
+    """Host-side inputs of the oracle for a workload (drawn once per process: the vocabulary weights alone take seconds)."""
+    import torch
+    from paper_2603_24840_b200 import synth
+    if w.name not in _ORACLE_INPUTS:
+        ell = synth.lengths(w)
+        off = synth.src_offsets(ell)
+        hist_s, hist_y = synth.calib_history(w)
+        _ORACLE_INPUTS[w.name] = dict(
+            ell=ell, off=off, rew=synth.rewards(w), head=synth.head_weights(w), tokens=synth.token_ids(w, int(off[-1])),
+            hist_s=hist_s, hist_y=hist_y, Wv=synth.as_oracle_array(synth.vocab_weights(w, dtype=torch.bfloat16)))
+    return _ORACLE_INPUTS[w.name]
+
+
 def oracle_step_rate(w, budget_s: float, x_cut=None, logp_rows=None):
     """Times the oracle on the workload: head scoring, probability map, selection, scan, token gather and
     advantages at full size on the given cutoff rows; the fp64 log-softmax gather on a bounded sample of survivor
@@ -188,16 +205,12 @@ def oracle_step_rate(w, budget_s: float, x_cut=None, logp_rows=None):
     import oracle
     from paper_2603_24840_b200 import synth
 
-    ell = synth.lengths(w)
-    off = synth.src_offsets(ell)
-    rew = synth.rewards(w)
-    head = synth.head_weights(w)
-    tokens = synth.token_ids(w, int(off[-1]))
-    hist_s, hist_y = synth.calib_history(w)
+    inp = oracle_inputs(w)
+    ell, off, rew, head, tokens = inp["ell"], inp["off"], inp["rew"], inp["head"], inp["tokens"]
+    hist_s, hist_y, Wv = inp["hist_s"], inp["hist_y"], inp["Wv"]
     oa = lambda t: None if t is None else synth.as_oracle_array(t)
     if x_cut is None:
         x_cut = synth.hidden_states(w, w.N, stream=21)
-    Wv = oa(synth.vocab_weights(w, dtype=torch.bfloat16))
     cores = oracle.num_threads()
 
     t0 = time.perf_counter()
@@ -259,8 +272,8 @@ def run_reference(args, w):
     out = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(walls)) * 1e3,
-        "ms_per_step_note": "wall time of one bounded-sample step (input preparation included); the whole workload "
-                            "would take survivor_tokens / value seconds per step",
+        "ms_per_step_note": "wall time of one bounded-sample step; the whole workload would take survivor_tokens / value "
+                            "seconds per step",
         "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config_of(w, C),
@@ -292,6 +305,11 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
     stream = torch.cuda.current_stream()
     props = torch.cuda.get_device_properties(local)
     sm_count = props.multi_processor_count
+
+    # ---- scoring kernel on its own, before the long tensor-core runs (a kernel timed alone, at the clocks a short
+    # kernel gets; after seconds under the power cap the same call measures 20 % less) ----
+    views[0].step()
+    score = score_times(views[0], pr_full, w, B, torch, stream, K)
 
     for _ in range(W):
         for v in views:
@@ -342,18 +360,22 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
     # effective SM clock inside the last log-prob launch, and the tensor-pipe fraction at that clock
     T_last = counts[-1][1]
     splits = B.arrol_token_logprob_splits(ctx, views[-1].cap, w.d, w.V)
-    items_last = ((T_last + 127) // 128) * splits
-    st = stamps.cpu().numpy().reshape(-1, 4)[:items_last]
+    tiles_last = (T_last + 127) // 128
+    st = stamps.cpu().numpy().reshape(-1, 4)
+    st = st[st[:, 1] > st[:, 0]]                 # the work items of the last launch that left a stamp
     in_kernel = None
-    if items_last > 0 and np.all(st[:, 1] > st[:, 0]):
+    if len(st) > 0:
+        # the kernel runs as pairs of blocks on 256-row tiles (one stamp per pair) or as single blocks
+        blocks_per_item = 2 if len(st) <= ((tiles_last + 1) // 2) * splits else 1
         ns = (st[:, 1] - st[:, 0]).astype(np.float64)
-        cyc = (st[:, 3] - st[:, 2]).astype(np.float64)
+        cyc = (st[:, 3] - st[:, 2]).astype(np.float64) * blocks_per_item
         span_ns = float(st[:, 1].max() - st[:, 0].min())
-        mhz = float(cyc.sum() / ns.sum() * 1e3)
+        mhz = float(cyc.sum() / ns.sum() * 1e3) / blocks_per_item
         flops_last = 2.0 * T_last * w.d * w.V
         in_kernel = {
             "sm_mhz": mhz, "what": "sum of SM cycles / sum of nanoseconds over the work items of the region's last "
                                    "log-prob launch (clock64 and globaltimer read by the kernel; no clock control touched)",
+            "blocks_per_work_item": blocks_per_item,
             "busy_cycles_per_sm": float(cyc.sum() / sm_count), "span_ms": span_ns / 1e6,
             "tensor_frac_at_clock": flops_last / (sm_count * 8192.0 * (span_ns * mhz * 1e-3)),
             "tensor_frac_of_busy_cycles": flops_last / (8192.0 * cyc.sum()),
@@ -389,9 +411,6 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
     if C > 1:
         prune_us["all_prompts"] = prune_step_times(pr_full, B, torch, stream, K, rows_too=False)
         prune_us["note"] = "per chunk of %d prompts; all_prompts: one call over all %d prompts" % (w.P // C, w.P)
-
-    # ---- scoring kernel on its own ----
-    score = score_times(views[0], pr_full, w, B, torch, stream, K)
 
     update = aux = None
     if full and not args.skip_update:

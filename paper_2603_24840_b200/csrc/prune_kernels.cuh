@@ -51,36 +51,11 @@ template <> struct Vec16<__nv_bfloat16> {
     }
 };
 
-// Dot product of one hidden row with the linear head's weights by one warp (Section 4.2): 16-byte loads, eight of x
-// and eight of w in flight per lane (a 4 KB row is one round trip), four accumulators per lane, shuffle reduction.
-// Every lane returns the row's sum (without the bias).  nvec = d / Vec16<T>::N, or 0 to skip the row (sum 0).
-template <typename T>
-__device__ __forceinline__ float linear_row_dot(const T* __restrict__ x, const T* __restrict__ w, int nvec, int lane) {
-    constexpr int VN = Vec16<T>::N;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int c0 = lane; c0 < nvec; c0 += 256) {
-        typename Vec16<T>::Raw xr[8], wr[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int c = c0 + 32 * u;
-            if (c < nvec) {
-                xr[u] = Vec16<T>::load_raw(x + (int64_t)c * VN);
-                wr[u] = Vec16<T>::load_raw(w + (int64_t)c * VN);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (c0 + 32 * u < nvec) acc[u & 3] = Vec16<T>::dot(xr[u], wr[u], acc[u & 3]);
-    }
-    float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    return s;
-}
-
-// The same reduction with the head's weights staged in shared memory (w_s: the d / VN 16-byte vectors of w): only the
-// row's own loads are in flight in registers, which is what a 1024-thread block can afford.  Products and sums are
-// taken in exactly the order of linear_row_dot, so the two give the same bits.
+// Dot product of one hidden row with the linear head's weights by one warp (Section 4.2) with the weights staged in
+// shared memory (w_s: the d / VN 16-byte vectors of w): 16-byte loads, eight of the row in flight per lane (a 4 KB row
+// is one round trip), four accumulators per lane, shuffle reduction; every lane returns the row's sum (without the
+// bias); nvec = d / Vec16<T>::N, or 0 to skip the row (sum 0).  Products and sums are taken in exactly the order of
+// score_linear_kernel, which keeps w's vectors in registers beside the row's, so the two give the same bits.
 template <typename T>
 __device__ __forceinline__ float linear_row_dot_ws(const T* __restrict__ x, const typename Vec16<T>::Raw* w_s, int nvec,
                                                    int lane) {

@@ -16,7 +16,10 @@
 
 namespace {
 
-template <typename T>
+// CHECK: the row numbers are range-checked against source_rows (arrol_set_source_rows); a separate instantiation, so
+// that the unchecked kernel keeps its 80 registers and six blocks per SM (with the check compiled in, 86-88 registers
+// and five blocks cost the streamed form of the kernel a tenth of its bandwidth)
+template <typename T, bool CHECK>
 __global__ void __launch_bounds__(128)
 score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int64_t* __restrict__ row_index, int N,
                     int d, const T* __restrict__ w, const T* __restrict__ bias, int B,
@@ -32,12 +35,36 @@ score_linear_kernel(const T* __restrict__ hidden, int64_t row_stride, const int6
     if (warp >= N) return;
     const int64_t row = row_index ? row_index[warp] : (int64_t)warp;
     const T* x = hidden + row * row_stride;
-    int nvec = d / VN;
-    if (source_rows > 0 && (row < 0 || row >= source_rows)) {   // outside the caller's buffer: never read, scored as zeros
-        if (lane == 0) atomicOr(d_status, ARROL_DEV_BAD_INDEX);
-        nvec = 0;
+    if constexpr (CHECK) {
+        if (row < 0 || row >= source_rows) {   // outside the caller's buffer: never read, scored as zeros
+            if (lane == 0) {
+                atomicOr(d_status, ARROL_DEV_BAD_INDEX);
+                probability_map(bias ? to_f32(bias[0]) : 0.f, warp, B, q_lut, score, prob, bin, q);
+            }
+            return;
+        }
     }
-    float s = linear_row_dot<T>(x, w, nvec, lane);
+    const int nvec = d / VN;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    // eight independent 16-byte loads of x (and of w) in flight per lane: a 4 KB row is one round trip.  (The fused
+    // prune step's linear_row_dot_ws takes the same products and sums in the same order with w in shared memory.)
+    for (int c0 = lane; c0 < nvec; c0 += 256) {
+        typename Vec16<T>::Raw xr[8], wr[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int c = c0 + 32 * u;
+            if (c < nvec) {
+                xr[u] = Vec16<T>::load_raw(x + (int64_t)c * VN);
+                wr[u] = Vec16<T>::load_raw(w + (int64_t)c * VN);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (c0 + 32 * u < nvec) acc[u & 3] = Vec16<T>::dot(xr[u], wr[u], acc[u & 3]);
+    }
+    float s = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     if (lane == 0) {
         if (bias) s += to_f32(bias[0]);
         probability_map(s, warp, B, q_lut, score, prob, bin, q);
@@ -238,7 +265,8 @@ int launch_score(arrol_ctx* ctx, const void* hidden, int64_t row_stride, const i
     if (head->h == 0) {
         const int warps_per_block = 4;
         const int blocks = (N + warps_per_block - 1) / warps_per_block;
-        ARROL_CUDA_OK(arrol_launch_pdl(score_linear_kernel<T>, dim3(blocks), dim3(32 * warps_per_block), 0, s, hid,
+        auto kernel = ctx->source_rows > 0 ? score_linear_kernel<T, true> : score_linear_kernel<T, false>;
+        ARROL_CUDA_OK(arrol_launch_pdl(kernel, dim3(blocks), dim3(32 * warps_per_block), 0, s, hid,
                                        row_stride, row_index, N, head->d, static_cast<const T*>(head->W1),
                                        static_cast<const T*>(head->b1), B, q_lut, score, prob, bin, q,
                                        ctx->source_rows, ctx->d_status));
