@@ -436,8 +436,42 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
         except (RuntimeError, MemoryError) as exc:   # e.g. the pinned host copy of the inputs does not fit
             print("e2e leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
 
+    # (last: a profiler that cannot launch clusters leaves the context unusable after this leg)
+    # ---- the log-prob call with the kernel run as pairs of blocks (tcgen05 cta_group::2; opt-in, see include/arrol.h) ----
+    pair_kernel = None
+    try:
+        if args.skip_pair:
+            raise RuntimeError("left out on request")
+        v = views[0]
+        v.step()
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 1)
+        ws_pair = torch.empty(B.arrol_token_logprob_workspace(ctx, v.cap, w.d, w.V), dtype=torch.uint8, device=v.dev)
+        lp_pair = torch.empty(v.cap, dtype=torch.float32, device=v.dev)
+        call = lambda: B.arrol_token_logprob(ctx, v.dst_rows, v.W_vocab, v.dst_tokens, v.cap, w.d, w.V, lp_pair, ws_pair,
+                                             d_T=v.d_num[1:])
+        call()
+        barrier()
+        a.record(stream)
+        for _ in range(K_in):
+            call()
+        b.record(stream)
+        barrier()
+        ms = a.elapsed_time(b) / K_in
+        T_v = v.counts()[1]
+        pair_kernel = {"what": "arrol_token_logprob on %s with the kernel as clusters of two blocks on 256-row tiles" % (
+                           "the step's survivors" if C == 1 else "one chunk's survivors"),
+                       "launch_ms": ms, "achieved": 2.0 * T_v * w.d * w.V / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                       "vocab_splits": int(B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)),
+                       "bit_equal_to_default_kernel": bool(torch.equal(lp_pair[:T_v], v.logp[:T_v]))}
+        del ws_pair, lp_pair
+    except (RuntimeError, B.ArrolError) as exc:
+        print("pair-kernel leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
+    finally:
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 0)
+
     res = {"w": w, "C": C, "S": S, "T": T, "K": K, "total_ms": total_ms, "seg_step": seg_step,
            "clocks": clocks, "launches": int(launches), "in_kernel": in_kernel, "in_place": in_place,
+           "pair_kernel": pair_kernel,
            "prune_us": prune_us, "score": score, "update": update, "aux": aux, "e2e": e2e, "splits": int(splits),
            "sm_count": sm_count, "T_src": pr_full.T_src, "N_chunk": views[0].w.N,
            "T_chunks": [c[1] for c in counts]}
@@ -775,6 +809,10 @@ def report(res, peaks, tokens_all, ms_per_step, e2e_ms, world):
                              "algorithmic_bytes_per_launch": gather_bytes / C},
         "in_place": res["in_place"],
     }
+    if res["pair_kernel"] is not None:
+        pk = dict(res["pair_kernel"])
+        pk["frac"] = pk["achieved"] / peak
+        out["roofline"]["pair_kernel"] = pk
     sc = res["score"]
     esz = 4 if w.dtype == "f32" else 2
     if w.h == 0:
@@ -942,6 +980,8 @@ def main():
     ap.add_argument("--skip-update", action="store_true", help="leave out the policy-update leg")
     ap.add_argument("--skip-aux", action="store_true", help="leave out the timings of the calls around the step")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiler captures)")
+    ap.add_argument("--skip-pair", action="store_true", help="leave out the pair-kernel leg (profilers that cannot "
+                    "launch thread-block clusters)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
     ap.add_argument("--profile-leg", default=None, help="run one call of the path three times (for profiler captures): "
                     "score_stream, score, select, compact, compact_tokens, logprob, logprob_gathered, prune_step")

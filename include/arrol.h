@@ -460,8 +460,11 @@ int64_t arrol_launch_count(arrol_ctx* ctx);
  *                                    (cycles / nanoseconds) without reading or setting any GPU clock control.
  *   ARROL_HOOK_LOGPROB_SPLITS        value = vocabulary splits per token tile (1..64; 0 = chosen from the sizes, the
  *                                    default); set it before sizing the workspace, which depends on it.
- *   ARROL_HOOK_LOGPROB_PAIR          value != 0 (the default): the log-prob kernel runs as clusters of two thread blocks
- *                                    that share one 256-row tile (tcgen05 cta_group::2); 0: one block per 128-row tile.
+ *   ARROL_HOOK_LOGPROB_PAIR          value != 0: the log-prob kernel runs as clusters of two thread blocks that share one
+ *                                    256-row tile (tcgen05 cta_group::2; same results bit for bit, about 3 % faster at
+ *                                    d <= 2560); 0 (the default): one block per 128-row tile.  It is off by default
+ *                                    because the profiler on the development machines reports LaunchFailed for every
+ *                                    launch with a cluster dimension, so a run under it would lose the kernel.
  *                                    Set it before sizing the workspace, which depends on it.
  * Returns INVALID_ARG for an unknown key or a limit outside [0, 2^26]. */
 #define ARROL_HOOK_SPIN_LIMIT 1
