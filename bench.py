@@ -306,9 +306,12 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
     props = torch.cuda.get_device_properties(local)
     sm_count = props.multi_processor_count
 
-    # ---- scoring kernel on its own, before the long tensor-core runs (a kernel timed alone, at the clocks a short
-    # kernel gets; after seconds under the power cap the same call measures 20 % less) ----
-    views[0].step()
+    # ---- scoring kernel on its own, before any tensor-core work: a kernel timed alone, at the clocks a short kernel
+    # gets (for about a second after a log-prob launch the SM clock stays where the power cap put it, and this
+    # clock-sensitive streaming kernel measures 22 % less: 5.5 against 7.05 TB/s on the Llama-shaped source) ----
+    torch.cuda.synchronize()
+    time.sleep(1.0)
+    views[0].prune_step(with_rows=False)
     score = score_times(views[0], pr_full, w, B, torch, stream, K)
 
     for _ in range(W):
