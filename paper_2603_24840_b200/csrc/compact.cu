@@ -130,6 +130,7 @@ gather_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_
 // Per-token outputs without a payload plane (token ids, survivor ordinal, advantage): one block per survivor walks
 // its run of tokens with coalesced 4-byte accesses, so nothing has to be searched.  Blocks past S return at once.
 constexpr int TOKENS_THREADS = 128;
+constexpr int TOKENS_PER_THREAD = 16;   // token ids in flight per thread (4: 28.7 us, 8: 26.4, 16: 24.6 for the Qwen-3-4B-shaped step)
 __global__ void __launch_bounds__(TOKENS_THREADS)
 gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_seqlens,
                      const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
@@ -148,15 +149,15 @@ gather_tokens_kernel(const int64_t* __restrict__ d_num, const int64_t* __restric
         const int len = (int)(__ldg(cu_seqlens + s + 1) - c0);
         const int64_t src0 = __ldg(src_tok_off + __ldg(survivor_idx + s));
         const float a = __ldg(adv + s);
-        for (int t0 = threadIdx.x; t0 < len; t0 += 4 * TOKENS_THREADS) {
-            int32_t tok[4];
+        for (int t0 = threadIdx.x; t0 < len; t0 += TOKENS_PER_THREAD * TOKENS_THREADS) {
+            int32_t tok[TOKENS_PER_THREAD];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < TOKENS_PER_THREAD; ++u) {
                 const int t = t0 + u * TOKENS_THREADS;
                 if (dst_tokens && t < len) tok[u] = __ldg(src_tokens + src0 + t);
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < TOKENS_PER_THREAD; ++u) {
                 const int t = t0 + u * TOKENS_THREADS;
                 if (t < len) {
                     if (dst_tokens) dst_tokens[c0 + t] = tok[u];
