@@ -479,3 +479,35 @@ def test_pairs_of_blocks_and_single_blocks_give_the_same_logprobs(T, d, V, split
     assert np.abs(out[0][0].cpu().numpy()[rows] - lp_ref).max() <= LOGP_TOL
     assert np.abs(out[0][1].cpu().numpy()[rows] - lse_ref).max() <= LOGP_TOL
     ctx.close()
+
+
+def test_logprob_call_replayed_from_a_cuda_graph():
+    """arrol_token_logprob allocates nothing and never synchronises: a launch of several waves (the wave counter is
+    cleared by a memset node, the kernel is launched cooperatively) can be captured once and replayed."""
+    ctx = B.Context(0)
+    g = np.random.default_rng(11)
+    T, d, V = 128 * 148 * 2 + 300, 64, 777
+    H = torch.from_numpy(g.normal(size=(T, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    W = torch.from_numpy(g.normal(0, 0.05, size=(V, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    y = dev(g.integers(0, V, size=T).astype(np.int32))
+    ws = torch.empty(B.arrol_token_logprob_workspace(ctx, T, d, V), dtype=torch.uint8, device="cuda")
+    ref = torch.full((T,), 7.0, device="cuda")
+    B.arrol_token_logprob(ctx, H, W, y, T, d, V, ref, ws)
+    torch.cuda.synchronize()
+    lp = torch.full((T,), 7.0, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        B.arrol_token_logprob(ctx, H, W, y, T, d, V, lp, ws, stream=side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        B.arrol_token_logprob(ctx, H, W, y, T, d, V, lp, ws, stream=side)
+    for _ in range(2):
+        lp.fill_(7.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(lp, ref)
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
+    del graph
+    ctx.close()

@@ -116,3 +116,34 @@ def test_back_to_back_steps_never_read_the_previous_steps_results():
             assert torch.equal(getattr(pr, k)[:T], want[k][:T]), k
     assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
     pr.ctx.close()
+
+
+@pytest.mark.parametrize("P,G,K", [(1, 1, 1), (7, 1, 1), (5, 3, 2), (9, 5, 1), (3, 32, 7), (40, 32, 16), (200, 4, 4), (333, 2, 1),
+                                   (150, 16, 8), (1000, 2, 1)])
+def test_fused_prune_step_over_group_shapes(P, G, K):
+    """Group sizes that are no power of two, one group per block and many, more blocks than one wave of the chained
+    scan would hold (the call then takes the three separate launches): always what the three calls give."""
+    import dataclasses
+    w = dataclasses.replace(synth.WORKLOADS["mini"], P=P, G=G, K=K, h=0, seed=100 + P + G)
+    pr = PruneRebatch(w, inputs=host_inputs(w), with_rows=False)
+    pr.prune_step(with_rows=False)
+    torch.cuda.synchronize()
+    keys = ("score", "prob", "q", "bin", "keep", "survivor_idx", "cu_seqlens", "adv", "d_num", "dst_tokens", "tok_adv", "tok_seq")
+    want = {k: getattr(pr, k).clone() for k in keys}
+    S, T = pr.counts()
+    assert S == P * K
+    for _ in range(2):                                  # twice: the chained scan's published totals are cleared in between
+        for k in keys:
+            getattr(pr, k).fill_(0)
+        B.arrol_prune_step(pr.ctx, pr.prune_step_args(with_rows=False))
+        torch.cuda.synchronize()
+        assert pr.counts() == (S, T)
+        for k in ("score", "prob", "q", "bin", "keep", "d_num"):
+            assert torch.equal(getattr(pr, k), want[k]), k
+        for k in ("survivor_idx", "adv"):
+            assert torch.equal(getattr(pr, k)[:S], want[k][:S]), k
+        assert torch.equal(pr.cu_seqlens[:S + 1], want["cu_seqlens"][:S + 1])
+        for k in ("dst_tokens", "tok_adv", "tok_seq"):
+            assert torch.equal(getattr(pr, k)[:T], want[k][:T]), k
+    assert B.arrol_poll_status(pr.ctx, raise_on_error=False) == 0
+    pr.ctx.close()
