@@ -40,7 +40,8 @@ constexpr int ARROL_MLP_TH = 64;             // hidden units per MLP thread-bloc
 constexpr int ARROL_MAX_H = 4096;
 constexpr size_t ARROL_SCRATCH_FLOATS = (size_t)ARROL_MAX_MLP_N * (ARROL_MAX_H / ARROL_MLP_TH);
 constexpr size_t ARROL_PACK_BYTES = (size_t)64 << 20;
-constexpr int ARROL_TILE_COUNTERS = 1024;   // [0, 512) row tiles of the MLP head, [1023] log-prob waves
+constexpr int ARROL_TILE_COUNTERS = 1024;   // [0, 1020) row tiles of the MLP head, [1023] log-prob waves
+constexpr int ARROL_SCORE_ROW_TILES = 1020;
 constexpr int ARROL_CHAIN_BLOCKS = 510;      // blocks of the fused prune step's chained scan (2 + 2 * 510 words = 8 KB)
 
 #define ARROL_CUDA_OK(expr)                      \
