@@ -524,7 +524,19 @@ def prune_step_times(pr, B, torch, stream, K, rows_too=True):
         b.record(stream)
         torch.cuda.synchronize()
         out["tokens_only_graph"] = a.elapsed_time(b) / reps * 1e3
-        del graph
+        # and with L2 flushed before every replay (a 256 MB fill), one replay per measurement: the step as it runs
+        # after other work has displaced its inputs (cold rows, lengths, rewards and head weights)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=pr.dev)
+        cold = []
+        for _ in range(reps):
+            flush.fill_(1)
+            a.record(stream)
+            graph.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            cold.append(a.elapsed_time(b) * 1e3)
+        out["tokens_only_graph_l2_flushed"] = float(np.median(cold))
+        del graph, flush
     except RuntimeError as exc:
         print("graph replay of the prune step skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
     return out
