@@ -447,6 +447,7 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
             raise RuntimeError("left out on request")
         v = views[0]
         v.step()
+        default_splits = B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)
         B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 1)
         ws_pair = torch.empty(B.arrol_token_logprob_workspace(ctx, v.cap, w.d, w.V), dtype=torch.uint8, device=v.dev)
         lp_pair = torch.empty(v.cap, dtype=torch.float32, device=v.dev)
@@ -465,7 +466,11 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
                            "the step's survivors" if C == 1 else "one chunk's survivors"),
                        "launch_ms": ms, "achieved": 2.0 * T_v * w.d * w.V / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                        "vocab_splits": int(B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)),
-                       "bit_equal_to_default_kernel": bool(torch.equal(lp_pair[:T_v], v.logp[:T_v]))}
+                       # bit-equal whenever both forms use the same number of vocabulary splits (the split count
+                       # fixes the order of the log-sum-exp merge); with other counts the difference is rounding
+                       "default_kernel_vocab_splits": int(default_splits),
+                       "bit_equal_to_default_kernel": bool(torch.equal(lp_pair[:T_v], v.logp[:T_v])),
+                       "max_abs_diff_to_default_kernel": float((lp_pair[:T_v] - v.logp[:T_v]).abs().max())}
         del ws_pair, lp_pair
     except (RuntimeError, B.ArrolError) as exc:
         print("pair-kernel leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)

@@ -6,7 +6,8 @@
 // and a second launch writes the per-token outputs.
 //   prune_fused_kernel   a block owns 32 / G whole groups (at most 32 rollouts, one warp each).  Linear head: every
 //                        warp scores its rollout (the row reduction and probability map of score_linear_kernel) and
-//                        leaves q in shared memory; MLP head: q comes from the scoring kernel that ran before.  One or
+//                        leaves q in shared memory; MLP head: q comes from the scoring kernel that ran before (blocks
+//                        of two warps then, always 32 / G groups each).  One or
 //                        two warps run the per-group selection (select_lanes, as select_kernel) and write the keep
 //                        flags.  The first warp then scans the block's rollouts (kept, kept length), publishes the
 //                        block's totals, adds up the totals of the blocks before it as they appear (a chained scan:
@@ -120,7 +121,7 @@ prune_fused_kernel(const FusedParams p) {
             }
         }
     } else {
-        if (warp < n_here && lane == 0) q_s[warp] = pdl_acquire(p.q)[first + warp];
+        if (threadIdx.x < n_here) q_s[threadIdx.x] = pdl_acquire(p.q)[first + threadIdx.x];
     }
     __syncthreads();
     // selection on the block's groups: a group per segment of `seg` lanes
@@ -257,6 +258,10 @@ extern "C" int arrol_prune_step(arrol_ctx* ctx, const arrol_prune_step_args* a, 
     while (gpb > 1 && (a->P + gpb - 1) / gpb < ctx->sm_count / 2) gpb = (gpb + 1) / 2;
     int threads = 32 * gpb * a->G;
     if (threads < 64) threads = 64;                          // warp 1 fetches the lengths and rewards
+    if (!linear) {                                           // nothing to score: two warps per block, full blocks
+        gpb = 32 / a->G;
+        threads = 64;
+    }
     const int64_t fused_blocks = ((int64_t)a->P + gpb - 1) / gpb;
     const size_t w_bytes = linear ? (size_t)a->head.d * (a->head.dtype == ARROL_F32 ? 4 : 2) : 0;
     // the chained scan needs every block resident: at most (SMs x blocks that fit an SM) blocks
