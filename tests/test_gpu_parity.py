@@ -511,3 +511,33 @@ def test_logprob_call_replayed_from_a_cuda_graph():
     assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
     del graph
     ctx.close()
+
+
+@pytest.mark.parametrize("T_live", [0, 1, 129, 148 * 128 + 5, 2 * 148 * 128 + 300])
+def test_logprob_device_side_count_below_a_capacity_of_several_waves(T_live):
+    """The launch is sized for T_max (more than two waves of token tiles, so the blocks are held in step), the live count
+    comes from device memory: fewer waves than the host planned, blocks without a work item, nothing written past T."""
+    ctx = B.Context(0)
+    g = np.random.default_rng(12)
+    T_max, d, V = 2 * 148 * 128 + 300, 64, 600
+    H = torch.from_numpy(g.normal(size=(T_max, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    W = torch.from_numpy(g.normal(0, 0.05, size=(V, d)).astype(np.float32)).to(torch.bfloat16).cuda()
+    y = dev(g.integers(0, V, size=T_max).astype(np.int32))
+    ws = torch.empty(B.arrol_token_logprob_workspace(ctx, T_max, d, V), dtype=torch.uint8, device="cuda")
+    full = torch.empty(T_max, device="cuda")
+    B.arrol_token_logprob(ctx, H, W, y, T_max, d, V, full, ws)
+    d_T = torch.tensor([T_live], dtype=torch.int64, device="cuda")
+    lp = torch.full((T_max,), 7.0, device="cuda")
+    lse = torch.full((T_max,), 7.0, device="cuda")
+    for _ in range(2):
+        B.arrol_token_logprob(ctx, H, W, y, T_max, d, V, lp, ws, lse=lse, d_T=d_T)
+    torch.cuda.synchronize()
+    assert torch.equal(lp[:T_live], full[:T_live])          # same tiles, same splits: the same bits
+    assert torch.all(lp[T_live:] == 7.0) and torch.all(lse[T_live:] == 7.0)
+    rows = np.unique(np.concatenate([[0, max(T_live - 1, 0)], g.integers(0, max(T_live, 1), size=6)]))[: max(min(T_live, 8), 0)]
+    if T_live:
+        ref, _ = oracle.token_logprob(synth.as_oracle_array(H[torch.from_numpy(rows).cuda()].cpu()),
+                                      synth.as_oracle_array(W.cpu()), y.cpu().numpy()[rows])
+        assert np.abs(lp.cpu().numpy()[rows] - ref).max() <= 2e-3
+    assert B.arrol_poll_status(ctx, raise_on_error=False) == 0
+    ctx.close()
