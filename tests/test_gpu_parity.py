@@ -97,6 +97,10 @@ def test_linear_head(ctx, N, d, dtype, use_lut, use_index):
     (1000, 1024, 128, torch.bfloat16),      # several 128-row tiles and K ranges on the tensor-core path
     (257, 200, 68, torch.bfloat16),         # d and h off the 64-wide tile edges
     (2048, 2048, 256, torch.bfloat16),      # the Qwen-3-1.7B-shaped head
+    (40, 64, 64, torch.bfloat16),           # one K step: three of the four MMA issuers have nothing to do
+    (33, 128, 16, torch.bfloat16),          # two K steps
+    (17, 8, 4, torch.bfloat16),             # a K step of 8 columns, 4 hidden units
+    (4096, 4096, 512, torch.bfloat16),      # the DAPO-shaped head over all prompts (256 blocks: more than one wave)
 ])
 def test_mlp_head(ctx, N, d, h, dtype):
     _score_case(ctx, N, d, h, dtype, True, True, seed=N + h)
