@@ -439,19 +439,19 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
         except (RuntimeError, MemoryError) as exc:   # e.g. the pinned host copy of the inputs does not fit
             print("e2e leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
 
-    # (last: a profiler that cannot launch clusters leaves the context unusable after this leg)
-    # ---- the log-prob call with the kernel run as pairs of blocks (tcgen05 cta_group::2; opt-in, see include/arrol.h) ----
-    pair_kernel = None
+    # ---- the log-prob call with the kernel's other form: one block per 128-row tile instead of pairs of blocks on
+    # 256-row tiles (tcgen05 cta_group::2, the default; see include/arrol.h, ARROL_HOOK_LOGPROB_PAIR) ----
+    single_kernel = None
     try:
         if args.skip_pair:
             raise RuntimeError("left out on request")
         v = views[0]
         v.step()
         default_splits = B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)
-        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 1)
-        ws_pair = torch.empty(B.arrol_token_logprob_workspace(ctx, v.cap, w.d, w.V), dtype=torch.uint8, device=v.dev)
-        lp_pair = torch.empty(v.cap, dtype=torch.float32, device=v.dev)
-        call = lambda: B.arrol_token_logprob(ctx, v.dst_rows, v.W_vocab, v.dst_tokens, v.cap, w.d, w.V, lp_pair, ws_pair,
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 0)
+        ws_alt = torch.empty(B.arrol_token_logprob_workspace(ctx, v.cap, w.d, w.V), dtype=torch.uint8, device=v.dev)
+        lp_alt = torch.empty(v.cap, dtype=torch.float32, device=v.dev)
+        call = lambda: B.arrol_token_logprob(ctx, v.dst_rows, v.W_vocab, v.dst_tokens, v.cap, w.d, w.V, lp_alt, ws_alt,
                                              d_T=v.d_num[1:])
         call()
         barrier()
@@ -462,24 +462,25 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
         barrier()
         ms = a.elapsed_time(b) / K_in
         T_v = v.counts()[1]
-        pair_kernel = {"what": "arrol_token_logprob on %s with the kernel as clusters of two blocks on 256-row tiles" % (
-                           "the step's survivors" if C == 1 else "one chunk's survivors"),
-                       "launch_ms": ms, "achieved": 2.0 * T_v * w.d * w.V / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                       "vocab_splits": int(B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)),
-                       # bit-equal whenever both forms use the same number of vocabulary splits (the split count
-                       # fixes the order of the log-sum-exp merge); with other counts the difference is rounding
-                       "default_kernel_vocab_splits": int(default_splits),
-                       "bit_equal_to_default_kernel": bool(torch.equal(lp_pair[:T_v], v.logp[:T_v])),
-                       "max_abs_diff_to_default_kernel": float((lp_pair[:T_v] - v.logp[:T_v]).abs().max())}
-        del ws_pair, lp_pair
+        single_kernel = {"what": "arrol_token_logprob on %s with one block per 128-row tile (tcgen05 cta_group::1) instead "
+                                 "of the default pairs of blocks on 256-row tiles" % (
+                                     "the step's survivors" if C == 1 else "one chunk's survivors"),
+                         "launch_ms": ms, "achieved": 2.0 * T_v * w.d * w.V / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                         "vocab_splits": int(B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)),
+                         # bit-equal whenever both forms use the same number of vocabulary splits (the split count
+                         # fixes the order of the log-sum-exp merge); with other counts the difference is rounding
+                         "default_kernel_vocab_splits": int(default_splits),
+                         "bit_equal_to_default_kernel": bool(torch.equal(lp_alt[:T_v], v.logp[:T_v])),
+                         "max_abs_diff_to_default_kernel": float((lp_alt[:T_v] - v.logp[:T_v]).abs().max())}
+        del ws_alt, lp_alt
     except (RuntimeError, B.ArrolError) as exc:
-        print("pair-kernel leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
+        print("single-block-kernel leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
     finally:
-        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 0)
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 1)
 
     res = {"w": w, "C": C, "S": S, "T": T, "K": K, "total_ms": total_ms, "seg_step": seg_step,
            "clocks": clocks, "launches": int(launches), "in_kernel": in_kernel, "in_place": in_place,
-           "pair_kernel": pair_kernel,
+           "single_kernel": single_kernel,
            "prune_us": prune_us, "score": score, "update": update, "aux": aux, "e2e": e2e, "splits": int(splits),
            "sm_count": sm_count, "T_src": pr_full.T_src, "N_chunk": views[0].w.N,
            "T_chunks": [c[1] for c in counts]}
@@ -796,7 +797,7 @@ def report(res, peaks, tokens_all, ms_per_step, e2e_ms, world):
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     traffic, traffic_src = logprob_traffic(w, T / C, res["splits"], res["sm_count"])
     roofline = {
-        "kernel": "token_logprob_kernel (+ combine_splits_kernel)", "bound": "tensor", "achieved": achieved, "peak": peak,
+        "kernel": "token_logprob_kernel as pairs of blocks, tcgen05 cta_group::2 (+ combine_splits_kernel)", "bound": "tensor", "achieved": achieved, "peak": peak,
         "unit": "TFLOP/s", "frac": achieved / peak,
         "peak_source": "%s bf16 sustained (kernel timed inside a long step)" % peaks["source"],
         "frac_of_burst": achieved / float(peaks["bf16_tflops"]), "frac_of_nominal_2250": achieved / 2250.0,
@@ -829,10 +830,10 @@ def report(res, peaks, tokens_all, ms_per_step, e2e_ms, world):
                              "algorithmic_bytes_per_launch": gather_bytes / C},
         "in_place": res["in_place"],
     }
-    if res["pair_kernel"] is not None:
-        pk = dict(res["pair_kernel"])
+    if res["single_kernel"] is not None:
+        pk = dict(res["single_kernel"])
         pk["frac"] = pk["achieved"] / peak
-        out["roofline"]["pair_kernel"] = pk
+        out["roofline"]["single_block_kernel"] = pk
     sc = res["score"]
     esz = 4 if w.dtype == "f32" else 2
     if w.h == 0:
@@ -1000,8 +1001,8 @@ def main():
     ap.add_argument("--skip-update", action="store_true", help="leave out the policy-update leg")
     ap.add_argument("--skip-aux", action="store_true", help="leave out the timings of the calls around the step")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiler captures)")
-    ap.add_argument("--skip-pair", action="store_true", help="leave out the pair-kernel leg (profilers that cannot "
-                    "launch thread-block clusters)")
+    ap.add_argument("--skip-pair", action="store_true", help="leave out the leg that times the log-prob kernel's "
+                    "one-block form")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
     ap.add_argument("--profile-leg", default=None, help="run one call of the path three times (for profiler captures): "
                     "score_stream, score, select, compact, compact_tokens, logprob, logprob_gathered, prune_step")

@@ -49,7 +49,8 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->gather_bulk_smem_set = false;
     ctx->test_spin_limit = 0;
     ctx->test_mute_producer = 0;
-    ctx->logprob_pair = 0;
+    ctx->logprob_pair = 1;
+    for (int i = 0; i < 3; ++i) ctx->pair_max_clusters[i] = 0;
     ctx->logprob_splits = 0;
     ctx->logprob_timing = nullptr;
     ctx->logprob_timing_items = 0;

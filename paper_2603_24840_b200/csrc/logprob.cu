@@ -643,33 +643,56 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
     ARROL_CUDA_OK(cudaFuncSetAttribute(token_logprob_kernel<true, false, true>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     const int64_t m_tiles = (T_max + BM - 1) / BM;
+    typedef void (*KernelFn)(CUtensorMap, CUtensorMap, CUtensorMap, LogprobParams);
+    const int variant = ga ? 2 : (conf ? 1 : 0);
+    KernelFn fn;
+    if (pair) fn = ga ? token_logprob_kernel<false, true, true> : (conf ? token_logprob_kernel<true, false, true>
+                                                                         : token_logprob_kernel<false, false, true>);
+    else fn = ga ? token_logprob_kernel<false, true, false> : (conf ? token_logprob_kernel<true, false, false>
+                                                                     : token_logprob_kernel<false, false, false>);
     // work items and the units that take them: blocks, or pairs of blocks on 256 rows
     const int64_t items_max = (pair ? (m_tiles + 1) / 2 : m_tiles) * p.splits;
     int64_t units = pair ? ctx->sm_count / 2 : ctx->sm_count;
-    if (units > items_max) units = items_max;
-    const int64_t grid = pair ? 2 * units : units;
-    // more than one wave: the blocks wait for one another, so they must all be resident (cooperative launch)
-    const bool several_waves = items_max > units;
-    if (several_waves) ARROL_CUDA_OK(cudaMemsetAsync(p.wave_counter, 0, sizeof(unsigned int), s));
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(NUM_THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
     cudaLaunchAttribute attr[2];
     int n_attr = 0;
-    if (several_waves) {
-        attr[n_attr].id = cudaLaunchAttributeCooperative;
-        attr[n_attr].val.cooperative = 1;
-        ++n_attr;
-    }
     if (pair) {
         attr[n_attr].id = cudaLaunchAttributeClusterDimension;
         attr[n_attr].val.clusterDim.x = 2;
         attr[n_attr].val.clusterDim.y = 1;
         attr[n_attr].val.clusterDim.z = 1;
         ++n_attr;
+        // Pairs that wait for one another per wave must all be resident.  The cooperative attribute would have the
+        // driver check that, but the profiler cannot launch a cooperative grid of clusters that fills the GPU
+        // ("LaunchFailed"; the same grid without the attribute profiles), so the check is made here instead: never
+        // more pairs than the occupancy query says fit at once (asked once per context and kernel variant).  The
+        // waits themselves are bounded either way.
+        if (ctx->pair_max_clusters[variant] == 0) {
+            cfg.gridDim = dim3((unsigned)(2 * units));
+            cfg.attrs = attr;
+            cfg.numAttrs = n_attr;
+            int fit = 0;
+            ARROL_CUDA_OK(cudaOccupancyMaxActiveClusters(&fit, fn, &cfg));
+            if (fit < 1) return ARROL_ERR_CUDA;
+            ctx->pair_max_clusters[variant] = fit;
+        }
+        if (units > ctx->pair_max_clusters[variant]) units = ctx->pair_max_clusters[variant];
     }
+    if (units > items_max) units = items_max;
+    const int64_t grid = pair ? 2 * units : units;
+    // more than one wave: the blocks wait for one another, so they must all be resident (single blocks: cooperative
+    // launch)
+    const bool several_waves = items_max > units;
+    if (several_waves) ARROL_CUDA_OK(cudaMemsetAsync(p.wave_counter, 0, sizeof(unsigned int), s));
+    if (several_waves && !pair) {
+        attr[n_attr].id = cudaLaunchAttributeCooperative;
+        attr[n_attr].val.cooperative = 1;
+        ++n_attr;
+    }
+    cfg.gridDim = dim3((unsigned)grid);
     cfg.attrs = attr;
     cfg.numAttrs = n_attr;
     if (ga) {
@@ -678,16 +701,8 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
                                        static_cast<const uint4*>(hidden), ga->cu_seqlens, ga->survivor_idx,
                                        ga->src_tok_off, ga->d_num, ga->S_max, T_max, d / 8, static_cast<uint4*>(scratch)));
         ctx->launches += 1;
-        if (pair) ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, true, true>, map_h, map_s, map_w, p));
-        else ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, true, false>, map_h, map_s, map_w, p));
-    } else if (conf) {
-        if (pair) ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<true, false, true>, map_h, map_s, map_w, p));
-        else ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<true, false, false>, map_h, map_s, map_w, p));
-    } else if (pair) {
-        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, false, true>, map_h, map_s, map_w, p));
-    } else {
-        ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, token_logprob_kernel<false, false, false>, map_h, map_s, map_w, p));
     }
+    ARROL_CUDA_OK(cudaLaunchKernelEx(&cfg, fn, map_h, map_s, map_w, p));
     ctx->launches += 1;
     ARROL_CUDA_OK(cudaGetLastError());
     if (p.splits > 1) {
