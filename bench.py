@@ -34,7 +34,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic of one token_logprob launch per survivor token, by (d, V, vocabulary splits), from a single-launch
 # profiler capture on the small Llama-shaped case: (bytes read + bytes written) / tokens of the launch.  At fixed
 # d, V and split count the traffic grows in proportion to the tokens of the launch.
-LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256, 2): 60016.0}
+LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256, 2): 60090.0}
 # DRAM bytes per scored row of score_linear_kernel streamed over consecutive rows (same kind of capture)
 SCORE_LINEAR_DRAM_BYTES_PER_ROW = {(2048, 2): 4129.8}
 
@@ -439,16 +439,18 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
         except (RuntimeError, MemoryError) as exc:   # e.g. the pinned host copy of the inputs does not fit
             print("e2e leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
 
-    # ---- the log-prob call with the kernel's other form: one block per 128-row tile instead of pairs of blocks on
-    # 256-row tiles (tcgen05 cta_group::2, the default; see include/arrol.h, ARROL_HOOK_LOGPROB_PAIR) ----
-    single_kernel = None
+    # ---- the log-prob call with the kernel's OTHER form.  The library runs the kernel as pairs of blocks on 256-row
+    # tiles (tcgen05 cta_group::2) where pairs need no more vocabulary splits than single blocks, else as one block per
+    # 128-row tile (see include/arrol.h, ARROL_HOOK_LOGPROB_PAIR); this leg forces the form the step did not use ----
+    other_kernel = None
+    kernel_form = int(B.arrol_token_logprob_form(ctx, views[0].cap, w.d, w.V))
     try:
         if args.skip_pair:
             raise RuntimeError("left out on request")
         v = views[0]
         v.step()
         default_splits = B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)
-        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 0)
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 0 if kernel_form == 2 else 1)
         ws_alt = torch.empty(B.arrol_token_logprob_workspace(ctx, v.cap, w.d, w.V), dtype=torch.uint8, device=v.dev)
         lp_alt = torch.empty(v.cap, dtype=torch.float32, device=v.dev)
         call = lambda: B.arrol_token_logprob(ctx, v.dst_rows, v.W_vocab, v.dst_tokens, v.cap, w.d, w.V, lp_alt, ws_alt,
@@ -462,25 +464,28 @@ def measure(w, C, K, W, local, barrier, rank, full, args):
         barrier()
         ms = a.elapsed_time(b) / K_in
         T_v = v.counts()[1]
-        single_kernel = {"what": "arrol_token_logprob on %s with one block per 128-row tile (tcgen05 cta_group::1) instead "
-                                 "of the default pairs of blocks on 256-row tiles" % (
-                                     "the step's survivors" if C == 1 else "one chunk's survivors"),
-                         "launch_ms": ms, "achieved": 2.0 * T_v * w.d * w.V / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
-                         "vocab_splits": int(B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)),
-                         # bit-equal whenever both forms use the same number of vocabulary splits (the split count
-                         # fixes the order of the log-sum-exp merge); with other counts the difference is rounding
-                         "default_kernel_vocab_splits": int(default_splits),
-                         "bit_equal_to_default_kernel": bool(torch.equal(lp_alt[:T_v], v.logp[:T_v])),
-                         "max_abs_diff_to_default_kernel": float((lp_alt[:T_v] - v.logp[:T_v]).abs().max())}
+        other_kernel = {"what": "arrol_token_logprob on %s with the kernel forced to its other form: %s" % (
+                            "the step's survivors" if C == 1 else "one chunk's survivors",
+                            "one block per 128-row tile (tcgen05 cta_group::1)" if kernel_form == 2 else
+                            "pairs of blocks on 256-row tiles (tcgen05 cta_group::2)"),
+                        "launch_ms": ms, "achieved": 2.0 * T_v * w.d * w.V / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                        "vocab_splits": int(B.arrol_token_logprob_splits(ctx, v.cap, w.d, w.V)),
+                        # bit-equal whenever both forms use the same number of vocabulary splits (the split count
+                        # fixes the order of the log-sum-exp merge); with other counts the difference is rounding
+                        "default_kernel_vocab_splits": int(default_splits),
+                        "bit_equal_to_default_kernel": bool(torch.equal(lp_alt[:T_v], v.logp[:T_v])),
+                        "max_abs_diff_to_default_kernel": float((lp_alt[:T_v] - v.logp[:T_v]).abs().max()),
+                        "note": "a short leg at the end of the run: compare it with the figures of other short legs, not "
+                                "with the long timed region (the power cap settles lower over seconds)"}
         del ws_alt, lp_alt
     except (RuntimeError, B.ArrolError) as exc:
-        print("single-block-kernel leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
+        print("other-form leg skipped: %s" % str(exc).splitlines()[0], file=sys.stderr)
     finally:
-        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 1)
+        B.arrol_test_hook(ctx, B.HOOK_LOGPROB_PAIR, 2)
 
     res = {"w": w, "C": C, "S": S, "T": T, "K": K, "total_ms": total_ms, "seg_step": seg_step,
            "clocks": clocks, "launches": int(launches), "in_kernel": in_kernel, "in_place": in_place,
-           "single_kernel": single_kernel,
+           "other_kernel": other_kernel, "kernel_form": kernel_form,
            "prune_us": prune_us, "score": score, "update": update, "aux": aux, "e2e": e2e, "splits": int(splits),
            "sm_count": sm_count, "T_src": pr_full.T_src, "N_chunk": views[0].w.N,
            "T_chunks": [c[1] for c in counts]}
@@ -797,7 +802,9 @@ def report(res, peaks, tokens_all, ms_per_step, e2e_ms, world):
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     traffic, traffic_src = logprob_traffic(w, T / C, res["splits"], res["sm_count"])
     roofline = {
-        "kernel": "token_logprob_kernel as pairs of blocks, tcgen05 cta_group::2 (+ combine_splits_kernel)", "bound": "tensor", "achieved": achieved, "peak": peak,
+        "kernel": "token_logprob_kernel, %s (+ combine_splits_kernel)" % (
+            "pairs of blocks on 256-row tiles, tcgen05 cta_group::2" if res["kernel_form"] == 2 else
+            "one block per 128-row tile, tcgen05 cta_group::1"), "bound": "tensor", "achieved": achieved, "peak": peak,
         "unit": "TFLOP/s", "frac": achieved / peak,
         "peak_source": "%s bf16 sustained (kernel timed inside a long step)" % peaks["source"],
         "frac_of_burst": achieved / float(peaks["bf16_tflops"]), "frac_of_nominal_2250": achieved / 2250.0,
@@ -830,10 +837,10 @@ def report(res, peaks, tokens_all, ms_per_step, e2e_ms, world):
                              "algorithmic_bytes_per_launch": gather_bytes / C},
         "in_place": res["in_place"],
     }
-    if res["single_kernel"] is not None:
-        pk = dict(res["single_kernel"])
+    if res["other_kernel"] is not None:
+        pk = dict(res["other_kernel"])
         pk["frac"] = pk["achieved"] / peak
-        out["roofline"]["single_block_kernel"] = pk
+        out["roofline"]["other_form"] = pk
     sc = res["score"]
     esz = 4 if w.dtype == "f32" else 2
     if w.h == 0:
@@ -1002,7 +1009,7 @@ def main():
     ap.add_argument("--skip-aux", action="store_true", help="leave out the timings of the calls around the step")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg (profiler captures)")
     ap.add_argument("--skip-pair", action="store_true", help="leave out the leg that times the log-prob kernel's "
-                    "one-block form")
+                    "other form")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle log-prob work to time")
     ap.add_argument("--profile-leg", default=None, help="run one call of the path three times (for profiler captures): "
                     "score_stream, score, select, compact, compact_tokens, logprob, logprob_gathered, prune_step")

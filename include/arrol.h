@@ -157,6 +157,10 @@ int arrol_compact(arrol_ctx* ctx, const uint8_t* keep, const int32_t* lengths, c
 size_t arrol_token_logprob_workspace(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
 /* Number of vocabulary splits a launch on T_max tokens uses (1 = every block walks the whole vocabulary). */
 int32_t arrol_token_logprob_splits(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
+/* Form of the kernel for these sizes: 2 = pairs of thread blocks on 256-row token tiles (tcgen05 cta_group::2), 1 = one
+ * block per 128-row tile.  Pairs are used wherever they need no more vocabulary splits than single blocks (hidden
+ * widths up to about 2,700 on a 148-SM part); see ARROL_HOOK_LOGPROB_PAIR.  0 for invalid arguments. */
+int32_t arrol_token_logprob_form(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V);
 int arrol_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_vocab, const int32_t* targets,
                         int64_t T_max, const int64_t* d_T, int32_t d, int32_t V, float inv_temperature,
                         float* logp, float* lse, void* workspace, size_t workspace_bytes, void* stream);
@@ -460,12 +464,15 @@ int64_t arrol_launch_count(arrol_ctx* ctx);
  *                                    (cycles / nanoseconds) without reading or setting any GPU clock control.
  *   ARROL_HOOK_LOGPROB_SPLITS        value = vocabulary splits per token tile (1..64; 0 = chosen from the sizes, the
  *                                    default); set it before sizing the workspace, which depends on it.
- *   ARROL_HOOK_LOGPROB_PAIR          value != 0: the log-prob kernel runs as clusters of two thread blocks that share one
- *                                    256-row tile (tcgen05 cta_group::2; same results bit for bit, about 3 % faster at
- *                                    d <= 2560); 0 (the default): one block per 128-row tile.  It is off by default
- *                                    because the profiler on the development machines reports LaunchFailed for every
- *                                    launch with a cluster dimension, so a run under it would lose the kernel.
- *                                    Set it before sizing the workspace, which depends on it.
+ *   ARROL_HOOK_LOGPROB_PAIR          form of the log-prob kernel.  0: one thread block per 128-row token tile (tcgen05
+ *                                    cta_group::1, cooperative launch).  1: clusters of two thread blocks that share
+ *                                    one 256-row tile (tcgen05 cta_group::2; the same results bit for bit at equal
+ *                                    split counts, 1.5-3 % faster at equal split counts).  2 (the default): pairs where
+ *                                    they need no more vocabulary splits than single blocks, single blocks elsewhere
+ *                                    (with more splits the pairs draw more power and, under the board's power cap,
+ *                                    end up slower in long runs).  Pairs wait for one another per wave, so no more
+ *                                    of them are launched than cudaOccupancyMaxActiveClusters says are resident at
+ *                                    once (asked once per context).  Set it before sizing the workspace.
  * Returns INVALID_ARG for an unknown key or a limit outside [0, 2^26]. */
 #define ARROL_HOOK_SPIN_LIMIT 1
 #define ARROL_HOOK_MUTE_LOGPROB_PRODUCER 2

@@ -26,7 +26,7 @@ EXPORTS = [
     "arrol_calib_delta", "arrol_select_stochastic",
     "arrol_policy_loss", "arrol_lm_head_backward_workspace", "arrol_lm_head_backward", "arrol_rank_vote",
     "arrol_head_grad_workspace", "arrol_head_grad", "arrol_token_logprob_conf", "arrol_trace_confidence",
-    "arrol_prune_step", "arrol_token_logprob_splits", "arrol_test_hook", "arrol_set_source_rows",
+    "arrol_prune_step", "arrol_token_logprob_splits", "arrol_token_logprob_form", "arrol_test_hook", "arrol_set_source_rows",
     "arrol_token_logprob_gathered", "arrol_token_logprob_gathered_workspace",
 ]
 
@@ -260,6 +260,14 @@ def arrol_compact(ctx: Context, keep, lengths, src_tok_off, N: int, G: int, rewa
 
 def arrol_token_logprob_workspace(ctx: Context, T_max: int, d: int, V: int) -> int:
     return int(load_library().arrol_token_logprob_workspace(ctx.handle, int(T_max), int(d), int(V)))
+
+
+def arrol_token_logprob_form(ctx: Context, T_max: int, d: int, V: int) -> int:
+    """2 = the kernel runs as pairs of blocks on 256-row tiles for these sizes, 1 = one block per 128-row tile."""
+    lib = load_library()
+    lib.arrol_token_logprob_form.restype = C.c_int32
+    lib.arrol_token_logprob_form.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_int32]
+    return int(lib.arrol_token_logprob_form(ctx.handle, int(T_max), int(d), int(V)))
 
 
 def arrol_token_logprob_splits(ctx: Context, T_max: int, d: int, V: int) -> int:

@@ -24,7 +24,7 @@ struct arrol_ctx {
     unsigned long long* logprob_timing;   // arrol_test_hook: device buffer for per-work-item time stamps of the log-prob kernel
     int64_t logprob_timing_items;         // its capacity in work items (4 words each)
     int logprob_splits;        // arrol_test_hook: vocabulary splits of the log-prob kernel, 0 = chosen from the sizes
-    int logprob_pair;          // the log-prob kernel runs as clusters of two blocks (cta_group::2); arrol_test_hook switches it off
+    int logprob_pair;          // form of the log-prob kernel: 2 = pairs of blocks (cta_group::2) where they need no more splits (default), 1 = pairs, 0 = single blocks
     int pair_max_clusters[3];  // pairs of that kernel that are resident at once (plain, with confidence, rows in place); 0 = not asked yet
     int test_mute_producer;    // arrol_test_hook: the log-prob kernel's producer issues no copies (its waits run out)
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved once through the runtime

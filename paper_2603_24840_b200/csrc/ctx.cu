@@ -49,7 +49,7 @@ extern "C" int arrol_create(arrol_ctx** out, int device) {
     ctx->gather_bulk_smem_set = false;
     ctx->test_spin_limit = 0;
     ctx->test_mute_producer = 0;
-    ctx->logprob_pair = 1;
+    ctx->logprob_pair = 2;
     for (int i = 0; i < 3; ++i) ctx->pair_max_clusters[i] = 0;
     ctx->logprob_splits = 0;
     ctx->logprob_timing = nullptr;
@@ -132,7 +132,8 @@ extern "C" int arrol_test_hook(arrol_ctx* ctx, int32_t key, int64_t value) {
             ctx->logprob_splits = (int)value;
             return ARROL_OK;
         case ARROL_HOOK_LOGPROB_PAIR:
-            ctx->logprob_pair = value != 0;
+            if (value < 0 || value > 2) return ARROL_ERR_INVALID_ARG;
+            ctx->logprob_pair = (int)value;
             return ARROL_OK;
         case ARROL_HOOK_LOGPROB_TIMING_BUFFER:
             ctx->logprob_timing = reinterpret_cast<unsigned long long*>((uintptr_t)value);

@@ -2,8 +2,10 @@
 // (Section 3: log pi_theta(o_t | o_<t); Algorithm 1 "log-probs on R'"), as a fused contraction
 // hidden[T,d] x W_vocab[V,d]^T with an online max / log-sum-exp epilogue.  The T x V logits never leave the SM.
 //
-// One thread block per SM, persistent over work items (token tile of 128 rows, vocabulary split).  Per item the
-// block walks its vocabulary range in chunks of 256 columns.  Warp roles:
+// One thread block per SM, persistent over work items (token tile, vocabulary split).  By default the blocks work as
+// PAIRS (clusters of two, tcgen05 cta_group::2) on 256-row token tiles, see PAIR below; described first is the
+// one-block form on 128-row tiles, which the pair form extends.  Per item the block walks its vocabulary range in
+// chunks of 256 columns.  Warp roles:
 //   warp 0      TMA producer: K-major, 128-byte-swizzled tiles of hidden (128 x 64) and W_vocab (256 x 64) into
 //               a ring of shared-memory stages, completion on mbarriers
 //   warp 1      tcgen05.mma issuer (one elected lane): 128 x 256 x 16 bf16 MMAs into one of two 256-column fp32
@@ -19,8 +21,10 @@
 // its chunks from HBM, falls further behind, and the extra HBM traffic costs power: the SM clock under the 1 kW cap
 // fell from 1.40 GHz in the first waves to 0.72 GHz.  So the blocks are held in step: before issuing the loads of
 // wave k (its k-th work item) every producer arrives on a counter in global memory and waits until all blocks have
-// arrived for that wave.  The kernel is launched cooperatively whenever there is more than one wave, so that all
-// blocks are resident and the wait cannot deadlock; like every other wait it is bounded.
+// arrived for that wave.  All blocks must then be resident: single blocks are launched cooperatively whenever there is
+// more than one wave; for pairs the host asks cudaOccupancyMaxActiveClusters how many fit at once and launches no
+// more (a cooperative launch of clusters that fills the GPU is the one launch the profiler cannot make).  Like every
+// other wait this one is bounded.
 // Every wait is bounded; when one runs out the block records ARROL_DEV_WAIT_EXPIRED, drains and returns.
 //
 // Gathered variant (arrol_token_logprob_gathered; Section 4.3 (ii): the survivors are re-batched "to compute
@@ -508,7 +512,7 @@ __global__ void combine_splits_kernel(const PartialLse* __restrict__ partial, co
 // How many vocabulary splits per token tile.  With one split every resident block streams a different token
 // tile (128 x d x 2 bytes each) against the same W chunks; when those tiles together outgrow about half of L2
 // the tiles are re-fetched from HBM once per chunk, so the vocabulary is split until they fit.
-int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
+int splits_for(const arrol_ctx* ctx, int64_t T_max, int d, int V, bool pair) {
     const int total_chunks = (V + BN - 1) / BN;
     const int64_t m_tiles = (T_max + BM - 1) / BM;
     // Measured with the blocks in step (TFLOP/s, packed rows / rows read in place by the gathered variant):
@@ -524,15 +528,30 @@ int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
     // are scattered over the source buffer and 148 of them do not stay resident even at 74 MB), more only while the
     // resident tiles exceed 80 MB (one block per tile) or 50 MB (pairs).  The packed and the in-place variant follow
     // the same rule, so their results are bit-identical.
+    // Which form: pairs are 1.5-3 % faster at equal split counts; where they need more splits than single blocks
+    // (d = 4096: four against two) the extra W_vocab streams and the busier tensor pipe draw more power, and in a
+    // seconds-long run under the 1 kW cap the SM clock settles 4 % lower (1,195 against 1,250 MHz, read by the kernel)
+    // and the step is 2 % SLOWER (1,369 against 1,392-1,396 TFLOP/s).  So pairs only where they need no more splits.
     if (ctx->logprob_splits > 0) return ctx->logprob_splits < total_chunks ? ctx->logprob_splits : total_chunks;
     int splits = m_tiles >= ctx->sm_count ? 2 : 1;
-    const double l2_budget = (ctx->logprob_pair ? 50.0 : 80.0) * 1024 * 1024;
+    const double l2_budget = (pair ? 50.0 : 80.0) * 1024 * 1024;
     const double tile_bytes = (double)BM * d * 2;
     while (splits < 8 && (ctx->sm_count / splits) * tile_bytes > l2_budget) splits *= 2;
     // few token tiles: split so that every SM has work
     while (splits < 16 && m_tiles * splits < ctx->sm_count && splits * 2 <= total_chunks) splits *= 2;
     if (splits > total_chunks) splits = total_chunks;
     return splits < 1 ? 1 : splits;
+}
+
+// The form of the kernel for these sizes: pairs of blocks unless switched off, forced, or costlier in splits.
+bool pair_for(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
+    if (ctx->sm_count < 2 || ctx->logprob_pair == 0) return false;
+    if (ctx->logprob_pair == 1) return true;
+    return splits_for(ctx, T_max, d, V, true) <= splits_for(ctx, T_max, d, V, false);
+}
+
+int choose_splits(const arrol_ctx* ctx, int64_t T_max, int d, int V) {
+    return splits_for(ctx, T_max, d, V, pair_for(ctx, T_max, d, V));
 }
 
 }  // namespace
@@ -547,6 +566,11 @@ extern "C" size_t arrol_token_logprob_workspace(arrol_ctx* ctx, int64_t T_max, i
     size_t records = (size_t)(splits > 1 ? splits : 0) * (size_t)T_max;
     if (records < floor_records) records = floor_records;
     return records * sizeof(PartialLse) + 256;
+}
+
+extern "C" int32_t arrol_token_logprob_form(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
+    if (!ctx || T_max <= 0 || d <= 0 || V <= 0) return 0;
+    return pair_for(ctx, T_max, d, V) ? 2 : 1;
 }
 
 extern "C" int32_t arrol_token_logprob_splits(arrol_ctx* ctx, int64_t T_max, int32_t d, int32_t V) {
@@ -599,7 +623,7 @@ static int run_token_logprob(arrol_ctx* ctx, const void* hidden, const void* W_v
         map_s = map_h;
     }
     // pair variant (clusters of two blocks): every block loads half of a chunk's W_vocab rows
-    const bool pair = ctx->logprob_pair != 0 && ctx->sm_count >= 2;
+    const bool pair = pair_for(ctx, T_max, d, V);
     if (make_map(ctx, &map_w, W_vocab, (uint64_t)V, (uint64_t)d, pair ? PAIR_B_ROWS : BN) != ARROL_OK) return ARROL_ERR_CUDA;
 
     LogprobParams p;

@@ -456,7 +456,7 @@ def test_whole_path_mini():
 @pytest.mark.parametrize("T,d,V,splits", [(300, 64, 300, 0), (1000, 192, 3000, 0), (128 * 148 * 2 + 77, 64, 520, 0),
                                           (128 * 148 + 5, 64, 1100, 3), (700, 128, 2000, 2)])
 def test_pairs_of_blocks_and_single_blocks_give_the_same_logprobs(T, d, V, splits):
-    """The log-prob kernel as clusters of two blocks on 256-row tiles (opt-in) against one block per 128-row tile:
+    """The log-prob kernel as clusters of two blocks on 256-row tiles (the default) against one block per 128-row tile:
     the same products in the same order, so the same bits; both within 2e-3 of the oracle.  Covers a single partial
     wave, several waves (the blocks wait for one another per wave), an odd number of token tiles, forced splits."""
     ctx = B.Context(0)
@@ -487,7 +487,7 @@ def test_pairs_of_blocks_and_single_blocks_give_the_same_logprobs(T, d, V, split
 
 def test_logprob_call_replayed_from_a_cuda_graph():
     """arrol_token_logprob allocates nothing and never synchronises: a launch of several waves (the wave counter is
-    cleared by a memset node, the kernel is launched cooperatively) can be captured once and replayed."""
+    cleared by a memset node, a cluster launch) can be captured once and replayed."""
     ctx = B.Context(0)
     g = np.random.default_rng(11)
     T, d, V = 128 * 148 * 2 + 300, 64, 777
