@@ -1,8 +1,12 @@
 // Hidden-row plane of arrol_compact (Section 4.3 (ii): filter the pruned rollouts and re-batch the survivors) moved
 // by the copy engine: global -> shared -> global bulk copies (cp.async.bulk), so the payload never passes through
-// registers and one thread per role keeps a deep queue of 32 KB transfers in flight.
+// registers and one thread per role keeps a queue of 32 KB transfers in flight.
 //
-// One block per SM owns a contiguous run of destination tiles (as many whole rows as fit 32 KB).
+// Three blocks per SM, each with a ring of two stages (192 KB in flight per SM), own contiguous runs of destination
+// tiles (as many whole rows as fit 32 KB).  Measured: one block per SM with six stages 5,274 / 5,703 GB/s on the
+// Llama- / Qwen-3-4B-shaped steps, two blocks with three stages 5,288 / 5,708, three blocks with two stages
+// 5,540-5,562 / 6,036-6,082 (the same bytes in flight, more threads issuing copies), four blocks of two 24 KB stages
+// 5,473 / 6,114.  A ring needs at least two stages: a stage is freed when the NEXT store has been issued.
 //   thread 0 (producer)  for each tile: finds the survivors its rows belong to (binary search once, then a forward
 //                        walk in cu_seqlens) and issues one bulk load per contiguous source segment into a ring of
 //                        shared-memory stages; completion by transaction count on the stage's mbarrier
@@ -14,7 +18,9 @@
 
 namespace {
 
-constexpr int GB_STAGES = 6;
+constexpr int GB_STAGES = 2;
+constexpr int GB_BLOCKS_PER_SM = 3;
+static_assert(GB_STAGES >= 2, "the storer frees a stage only after it has issued the following store");
 constexpr int GB_TILE_BYTES = 32 * 1024;
 constexpr int GB_THREADS = 64;
 constexpr size_t GB_SMEM = (size_t)GB_STAGES * GB_TILE_BYTES + 1024 + 256;
@@ -39,7 +45,7 @@ __device__ __forceinline__ int find_survivor_of(const int64_t* __restrict__ cu_s
     return lo;
 }
 
-__global__ void __launch_bounds__(GB_THREADS, 1)
+__global__ void __launch_bounds__(GB_THREADS, GB_BLOCKS_PER_SM)
 gather_rows_bulk_kernel(const int64_t* __restrict__ d_num, const int64_t* __restrict__ cu_seqlens,
                         const int32_t* __restrict__ survivor_idx, const int64_t* __restrict__ src_tok_off,
                         const uint8_t* __restrict__ src_rows, int64_t row_bytes, int64_t capacity, int tile_rows,
@@ -146,7 +152,7 @@ int arrol_internal_gather_rows_bulk(arrol_ctx* ctx, const int64_t* d_num, const 
                                            (int)GB_SMEM));
         ctx->gather_bulk_smem_set = true;
     }
-    int64_t blocks = ctx->sm_count;
+    int64_t blocks = (int64_t)ctx->sm_count * GB_BLOCKS_PER_SM;
     if (blocks > max_tiles) blocks = max_tiles;
     if (blocks < 1) blocks = 1;
     ARROL_CUDA_OK(arrol_launch_pdl(gather_rows_bulk_kernel, dim3((unsigned)blocks), dim3(GB_THREADS), GB_SMEM, s, d_num,
