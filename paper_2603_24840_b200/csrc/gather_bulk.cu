@@ -150,6 +150,9 @@ int arrol_internal_gather_rows_bulk(arrol_ctx* ctx, const int64_t* d_num, const 
     if (!ctx->gather_bulk_smem_set) {
         ARROL_CUDA_OK(cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)GB_SMEM));
+        // all of the SM's shared memory, so that the three blocks fit side by side
+        ARROL_CUDA_OK(cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                           (int)cudaSharedmemCarveoutMaxShared));
         ctx->gather_bulk_smem_set = true;
     }
     int64_t blocks = (int64_t)ctx->sm_count * GB_BLOCKS_PER_SM;
