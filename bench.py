@@ -31,10 +31,11 @@ METRIC = "survivor_logprob_tokens_per_s"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "qwen3-8b-dapo"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM traffic of one token_logprob launch per survivor token, by (d, V, vocabulary splits), from a single-launch
-# profiler capture on the small Llama-shaped case: (bytes read + bytes written) / tokens of the launch.  At fixed
-# d, V and split count the traffic grows in proportion to the tokens of the launch.
-LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256, 2): 60090.0}
+# DRAM traffic of one token_logprob launch per survivor token, by (d, V, vocabulary splits), from single-launch
+# profiler captures on the small cases of the same d and V (the Llama-shaped and the DAPO-shaped one): (bytes read +
+# bytes written) / tokens of the launch.  At fixed d, V and split count the traffic grows in proportion to the tokens
+# of the launch.
+LOGPROB_DRAM_BYTES_PER_TOKEN = {(2048, 128256, 2): 60090.0, (4096, 151936, 2): 155108.0}
 # DRAM bytes per scored row of score_linear_kernel streamed over consecutive rows (same kind of capture)
 SCORE_LINEAR_DRAM_BYTES_PER_ROW = {(2048, 2): 4129.8}
 
@@ -45,7 +46,7 @@ def logprob_traffic(w, T, splits, sm_count):
     once and every token tile is read once per split."""
     per_tok = LOGPROB_DRAM_BYTES_PER_TOKEN.get((w.d, w.V, splits))
     if per_tok is not None:
-        return per_tok * T, "profiler capture on the small Llama-shaped case scaled by tokens"
+        return per_tok * T, "profiler capture on a small case of the same d, V and split count, scaled by tokens"
     return 2.0 * w.d * (splits + w.V * splits / (sm_count * 128.0)) * T, "model 2d(splits + V*splits/(SMs*128)) per token"
 
 

@@ -68,6 +68,9 @@ WORKLOADS: Dict[str, Workload] = {
         # Small case for profiler captures of the MLP head: the Qwen-3-1.7B-shaped N, d, h on short rollouts.
         Workload("profile-mlp", 128, 16, 8, 64, 128, ("uniform", 64, 128), 2048, 8192, "bf16", 256,
                  "beta_bernoulli", 10),
+        # Small case for profiler captures at the DAPO-shaped d, V and head: ~75k survivor tokens, about 3 GB on the device.
+        Workload("profile-wide", 48, 8, 4, 256, 512, ("uniform", 256, 512), 4096, 151936, "bf16", 512,
+                 "beta_bernoulli", 11),
         # Mid-size case for CPU-only tests: several tiles and ragged tails, seconds on the host.
         Workload("mini", 6, 8, 4, 16, 96, ("uniform", 16, 96), 192, 1000, "bf16", 24,
                  "beta_bernoulli", 7, degenerate_frac=0.34),
